@@ -1,0 +1,199 @@
+/*
+ * first.h -- C ABI of the router-selective decode step of FiRST (arXiv 2410.12513)
+ * for one NVIDIA B200 (sm_100a).
+ *
+ * The method (paper sections in quotes):
+ *   "Adaptive Router Module": before every transformer layer i sits a router R_i, a
+ *     bias-free linear map D -> 1.  It is applied to every prompt token's hidden state
+ *     entering layer i, a sigmoid is taken per token, and the mean over the sequence's
+ *     tokens is rho_i, the probability of running layer i for that sequence.
+ *   "Proposed Solution": at inference rho_i is rounded, keep = (rho_i >= 0.5), and
+ *     H_i = H_{i-1} + keep * phi_i(H_{i-1}) (Eq. 3 and the unnumbered inference rule):
+ *     a skipped layer is the identity on that sequence's residual stream.
+ *   "Inference for FiRST": (1) nothing is skipped during prefill; (2) the decisions
+ *     taken on the prompt are cached and every decode step obeys them, so a kept layer
+ *     always holds the K/V of all earlier tokens and a skipped layer needs none.
+ *
+ * This library is the decode-time hot path of that: score the routers on prefill hidden
+ * states (first_prefill_route), turn the per-sequence masks into per-layer lists of
+ * active rows (first_set_mask), and run decode steps in which each layer's kernels see
+ * only the rows that keep it (first_decode_step).
+ *
+ * General conventions
+ *   - Every function returns a status: 0 = FIRST_OK, negative = error; nothing throws.
+ *   - Pointers marked "dev" are device memory of the current CUDA device, "host" are
+ *     ordinary host memory.  All tensors are owned by the caller and only borrowed:
+ *     weights for the lifetime of the context, everything else for the call (the
+ *     kernels of a call may still be running on `stream` when it returns).
+ *   - The library allocates device memory only in first_create (its own scratch) and
+ *     frees it in first_destroy.
+ *   - Work is enqueued on the CUDA stream passed as `void *stream` (a cudaStream_t;
+ *     NULL = the default stream).  Only first_set_mask and first_last_device_flags
+ *     wait for the stream.
+ *   - Layers are numbered from 0.  mask[b][l] is a byte, 1 = sequence b runs layer l,
+ *     0 = it skips it.  All matrices are row-major; linear weights are [out][in].
+ *   - dtype FIRST_DTYPE_F32: weight matrices and KV cache are float32.
+ *     dtype FIRST_DTYPE_BF16: weight matrices and KV cache are bfloat16.
+ *     Norm gains, router weights, the residual stream and logits are always float32.
+ *   - Errors the host cannot see without a device read (cache slab full, token id out
+ *     of range, mask byte not 0/1, a bounded wait that ran out) set bits in a device
+ *     flag word; the offending row is left untouched.  first_last_device_flags reads it.
+ */
+#ifndef FIRST_H
+#define FIRST_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FIRST_OK 0
+#define FIRST_E_ARG (-1)         /* NULL pointer, negative size, value out of range */
+#define FIRST_E_SHAPE (-2)       /* sizes inconsistent with the model description */
+#define FIRST_E_UNSUPPORTED (-3) /* a shape or dtype the kernels do not cover */
+#define FIRST_E_CAPACITY (-4)    /* batch or token count beyond what the context was sized for */
+#define FIRST_E_CUDA (-5)        /* a CUDA runtime or driver call failed */
+#define FIRST_E_DEVICE_FLAG (-6) /* the device flag word is non-zero */
+#define FIRST_E_STATE (-7)       /* call order: e.g. decode before first_set_mask */
+
+#define FIRST_DTYPE_F32 0
+#define FIRST_DTYPE_BF16 1
+
+#define FIRST_FLAG_KV_FULL 1u      /* a kept (sequence, layer) had len == slab_cap */
+#define FIRST_FLAG_BAD_TOKEN 2u    /* token id outside [0, vocab) */
+#define FIRST_FLAG_BAD_MASK 4u     /* mask byte other than 0 or 1 */
+#define FIRST_FLAG_WAIT_EXPIRED 8u /* a bounded wait inside a kernel gave up */
+#define FIRST_FLAG_EMPTY_SEQ 16u   /* a router call saw a sequence with no tokens */
+
+#define FIRST_ROUTER_MEAN_OF_SIGMOID 0 /* the paper's order: rho = mean_j sigmoid(z_j) */
+#define FIRST_ROUTER_SIGMOID_OF_MEAN 1 /* pooled variant:    rho = sigmoid(mean_j z_j) */
+
+typedef struct first_ctx first_ctx;
+
+/* Decoder shape (the paper uses LLaMA-3 models; the block is the public LLaMA block:
+ * RMSNorm, rotary q/k with half-split pairing, grouped-query causal attention, SwiGLU). */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, ffn_dim, vocab;
+    float rope_base, rms_eps;
+    int32_t dtype;              /* FIRST_DTYPE_* */
+    int32_t max_batch;          /* largest B any later call will use */
+    int32_t max_tokens_per_seq; /* largest slab capacity of any sequence */
+} first_model_desc;
+
+/* Weights.  The pointer-array members are HOST arrays of n_layers DEVICE pointers. */
+typedef struct {
+    const void *embed;              /* dev [vocab][d_model]                         */
+    const void *lm_head;            /* dev [vocab][d_model]                         */
+    const float *final_norm;        /* dev [d_model]                                */
+    const float *const *attn_norm;  /* host[L] -> dev [d_model]                     */
+    const void *const *wqkv;        /* host[L] -> dev [(Hq+2*Hkv)*hd][d_model]: q rows, k rows, v rows */
+    const void *const *wo;          /* host[L] -> dev [d_model][Hq*hd]              */
+    const float *const *ffn_norm;   /* host[L] -> dev [d_model]                     */
+    const void *const *w_gate_up;   /* host[L] -> dev [2*ffn_dim][d_model]: gate rows, then up rows */
+    const void *const *w_down;      /* host[L] -> dev [d_model][ffn_dim]            */
+} first_weights;
+
+/* KV cache, caller-owned.  Layer l's keys are one tensor [Hkv][cap_total][hd]; sequence
+ * b owns token rows slab_off[b] .. slab_off[b]+slab_cap[b]-1 of every head ("ragged
+ * slabs").  len[l][b] tokens are present.  Item (2) of "Inference for FiRST": a kept
+ * (b,l) gains one token per step, a skipped (b,l) is neither read nor written and its
+ * len stays where prefill left it.  pos[b] is the absolute index of the token being
+ * fed (the rotary position), advanced by one per step for every sequence. */
+typedef struct {
+    void *const *k;          /* host[L] -> dev [Hkv][cap_total][hd] */
+    void *const *v;          /* host[L] -> dev [Hkv][cap_total][hd] */
+    const int64_t *slab_off; /* dev [B] */
+    const int32_t *slab_cap; /* dev [B] */
+    int32_t *len;            /* dev [L][B], updated by first_decode_step */
+    int32_t *pos;            /* dev [B],    updated by first_decode_step */
+    int64_t cap_total;       /* token rows per head in each layer tensor */
+} first_kv_cache;
+
+/* Create a context for one model on the current device: validates the description,
+ * borrows the weights, allocates scratch sized by max_batch / max_tokens_per_seq.
+ * Errors: FIRST_E_ARG, FIRST_E_SHAPE (head_dim*heads, divisibility), FIRST_E_UNSUPPORTED
+ * (head_dim not in {32,64,128}; Hq/Hkv not in {1,2,4,8}; d_model, ffn_dim not multiples
+ * of 8), FIRST_E_CUDA. */
+int first_create(const first_model_desc *desc, const first_weights *weights, first_ctx **out);
+int first_destroy(first_ctx *ctx);
+
+/* Router of ONE layer on that layer's prefill input ("Adaptive Router Module"; rounding
+ * rule of "Proposed Solution").  hidden holds the hidden states entering `layer` for all
+ * prompt tokens of a ragged batch, sequence b at rows cu_seqlens[b] .. cu_seqlens[b+1]-1.
+ *   z_j = router_w . hidden[j] (+ *router_b if router_b != NULL; the paper has no bias)
+ *   mode FIRST_ROUTER_MEAN_OF_SIGMOID: rho_b = mean_j sigmoid(z_j)
+ *   mode FIRST_ROUTER_SIGMOID_OF_MEAN: rho_b = sigmoid(mean_j z_j)
+ *   mask[b][layer] = (rho_b >= tau) ? 1 : 0   (equality keeps the layer), scores[b][layer] = rho_b.
+ * Token scores are float32, the per-sequence mean is taken in float64 in a fixed order,
+ * so the result does not depend on the launch shape.
+ *   ctx           required: it owns the per-token scratch the two passes share
+ *   hidden        dev [total_tokens][d_model], float32 or bfloat16 (hidden_dtype)
+ *   cu_seqlens    dev int32 [B+1], cu_seqlens[0] = 0, non-decreasing; every sequence needs
+ *                 at least one token (an empty one sets FIRST_FLAG_EMPTY_SEQ and its mask
+ *                 byte and score are left unwritten)
+ *   total_tokens  host value of cu_seqlens[B] (sizes the launch); at most
+ *                 max_batch*max_tokens_per_seq (the scratch capacity)
+ *   router_w      dev float32 [d_model];  router_b  dev float32 [1] or NULL
+ *   mask          dev uint8 [B][n_layers] (only column `layer` is written)
+ *   scores        dev float32 [B][n_layers] or NULL
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_CUDA. */
+int first_prefill_route(first_ctx *ctx, int32_t layer, const void *hidden, int32_t hidden_dtype,
+                        const int32_t *cu_seqlens, int32_t B, int64_t total_tokens, const float *router_w,
+                        const float *router_b, float tau, int32_t mode, uint8_t *mask, float *scores,
+                        void *stream);
+
+/* Fix the skip mask of the current batch and build, per layer, the ascending list of
+ * rows that keep it (one decision per sequence per layer, "Adaptive Router Module";
+ * fixed for all decode steps, "Inference for FiRST" item 2).  Must be called before
+ * first_decode_step and again whenever the batch or its mask changes.  Waits for the
+ * stream (the per-layer counts shape the later launches).
+ *   mask  dev uint8 [B][n_layers]
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY (B > max_batch), FIRST_E_DEVICE_FLAG (a mask byte
+ * other than 0/1), FIRST_E_CUDA. */
+int first_set_mask(first_ctx *ctx, const uint8_t *mask, int32_t B, void *stream);
+
+/* Read back the plan of the last first_set_mask (for inspection and tests).
+ *   idx   host int32 [n_layers][B]: idx[l][0..cnt[l]-1] ascending active rows, rest -1
+ *   cnt   host int32 [n_layers]
+ *   slot  host int32 [n_layers][B] or NULL: position of row b in idx[l], -1 if skipped */
+int first_get_plan(first_ctx *ctx, int32_t *idx, int32_t *cnt, int32_t *slot);
+
+/* One routed decode step for the whole batch (inference rule of "Proposed Solution";
+ * "Inference for FiRST" item 2).  For every sequence b: x = embed[tokens[b]]; for each
+ * layer l with mask[b][l] = 1: append the token's rotated key and value at row len[l][b]
+ * of its slab, attend over the len[l][b]+1 tokens, x += attention, x += SwiGLU FFN; layers
+ * with mask 0 leave x, the slab and len untouched.  logits[b] = lm_head . RMSNorm(x).
+ * Then pos[b] += 1.
+ *   tokens        dev int32 [B]
+ *   kv            host struct; see first_kv_cache
+ *   logits        dev float32 [B][vocab], or NULL
+ *   next_tokens   dev int32 [B] or NULL: argmax of the logits row, lowest index on ties
+ *   layer_inputs  dev float32 [n_layers][B][d_model] or NULL: the residual entering each
+ *                 layer (what router l reads when prompts are prefilled token by token
+ *                 with an all-keep mask)
+ * B is the batch of the last first_set_mask.
+ * Errors: FIRST_E_ARG, FIRST_E_STATE (no mask set), FIRST_E_CUDA; device flags for a full
+ * slab or a bad token id. */
+int first_decode_step(first_ctx *ctx, const int32_t *tokens, const first_kv_cache *kv, float *logits,
+                      int32_t *next_tokens, float *layer_inputs, void *stream);
+
+/* Wait for `stream`, read and clear the device flag word.  Returns FIRST_OK with
+ * *flags = 0, or FIRST_E_DEVICE_FLAG with the FIRST_FLAG_* bits in *flags. */
+int first_last_device_flags(first_ctx *ctx, uint32_t *flags, void *stream);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t first_launch_count(const first_ctx *ctx);
+
+/* Select kernel paths for A/B measurements.  Names: "max_gemv_rows" = largest active-row
+ * count served by the CUDA-core GEMV path (rows above it use the tensor-core path when
+ * the dtype is bfloat16); "attn_simple" = 1 forces the general attention kernel.  A
+ * negative value restores the default.  Errors: FIRST_E_ARG for an unknown name. */
+int first_set_option(first_ctx *ctx, const char *name, int64_t value);
+
+const char *first_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FIRST_H */

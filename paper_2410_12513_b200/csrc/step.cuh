@@ -1,0 +1,180 @@
+// Per-step kernels around the projections: embedding gather, RMSNorm of the compacted
+// active rows, rotary embedding + KV append, SwiGLU activation, greedy argmax.
+#pragma once
+#include "common.cuh"
+#include "first.h"
+
+namespace first {
+
+// Start of a step: residual rows from the embedding table, and the rotary cos/sin of
+// every sequence's position (same for all layers, so computed once, in float64:
+// angle = pos * base^(-2i/hd), half-split pairing).
+template <typename WT>
+__global__ void __launch_bounds__(256) step_begin(const int32_t* __restrict__ tokens, const WT* __restrict__ embed,
+                                                  int D, int V, const int32_t* __restrict__ pos,
+                                                  const double* __restrict__ inv_freq, int half,
+                                                  float* __restrict__ x, float2* __restrict__ cs,
+                                                  uint32_t* __restrict__ flags) {
+    const int b = blockIdx.x;
+    int tok = tokens[b];
+    if (tok < 0 || tok >= V) {
+        if (threadIdx.x == 0) atomicOr(flags, FIRST_FLAG_BAD_TOKEN);
+        tok = 0;
+    }
+    const WT* e = embed + (size_t)tok * D;
+    for (int k = threadIdx.x * 8; k < D; k += blockDim.x * 8) {
+        float f[8];
+        Load8<WT>::ld(e + k, f);
+        float4* o = reinterpret_cast<float4*>(x + (size_t)b * D + k);
+        o[0] = make_float4(f[0], f[1], f[2], f[3]);
+        o[1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    const double p = (double)pos[b];
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        double s, c;
+        sincos(p * inv_freq[i], &s, &c);
+        cs[(size_t)b * half + i] = make_float2((float)c, (float)s);
+    }
+}
+
+__device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16* hi, __nv_bfloat16* lo) {
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        h[e] = __float2bfloat16_rn(y[e]);
+        l[e] = __float2bfloat16_rn(y[e] - __bfloat162float(h[e]));
+    }
+    *reinterpret_cast<uint2*>(hi) = *reinterpret_cast<uint2*>(h);
+    *reinterpret_cast<uint2*>(lo) = *reinterpret_cast<uint2*>(l);
+}
+
+// RMSNorm of the rows a layer keeps, written compactly: out[i] = norm(x[idx[i]]) * gain.
+// Also emits the bfloat16 hi/lo split (v = hi + lo up to 2^-17 relative) that the
+// tensor-core projections consume, when asked.  One block per active row.
+__global__ void __launch_bounds__(256) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
+                                                    const float* __restrict__ gain, float eps, float* __restrict__ out,
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    __shared__ float red[8];
+    const int i = blockIdx.x;
+    const int b = idx ? idx[i] : i;
+    const float* xr = x + (size_t)b * D;
+    float ss = 0.f;
+    for (int k = threadIdx.x * 4; k < D; k += 1024) {
+        const float4 v = *reinterpret_cast<const float4*>(xr + k);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)D + eps);
+    for (int k = threadIdx.x * 4; k < D; k += 1024) {
+        const float4 v = *reinterpret_cast<const float4*>(xr + k);
+        const float4 g = *reinterpret_cast<const float4*>(gain + k);
+        const float y[4] = {v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w};
+        if (out) *reinterpret_cast<float4*>(out + (size_t)i * D + k) = make_float4(y[0], y[1], y[2], y[3]);
+        if (hi) split_store4(y, hi + (size_t)i * D + k, lo + (size_t)i * D + k);
+    }
+}
+
+// After the QKV projection: rotate q and k at the sequence's position, scale q by
+// 1/sqrt(hd), append k and v at row len[l][b] of the sequence's slab, len += 1.
+// qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  One block per active row.
+// A full slab sets FIRST_FLAG_KV_FULL and leaves cache and len alone.
+template <typename KT>
+__global__ void __launch_bounds__(256) rope_append(const float* __restrict__ qkv, const int32_t* __restrict__ idx,
+                                                   int Hq, int Hkv, int hd, const float2* __restrict__ cs,
+                                                   float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
+                                                   KT* __restrict__ vc, int64_t cap_total,
+                                                   const int64_t* __restrict__ slab_off,
+                                                   const int32_t* __restrict__ slab_cap, int32_t* __restrict__ len_l,
+                                                   uint32_t* __restrict__ flags) {
+    const int i = blockIdx.x, b = idx[i];
+    const int half = hd >> 1;
+    const int qd = Hq * hd, kvd = Hkv * hd;
+    const float* row = qkv + (size_t)i * (qd + 2 * kvd);
+    const float2* csb = cs + (size_t)b * half;
+    const int T = len_l[b];
+    const bool full = T >= slab_cap[b];
+    for (int p = threadIdx.x; p < Hq * half; p += blockDim.x) {
+        const int h = p / half, d = p - h * half;
+        const float2 c = csb[d];
+        const float a = row[h * hd + d], bb = row[h * hd + d + half];
+        q_out[(size_t)i * qd + h * hd + d] = (a * c.x - bb * c.y) * qscale;
+        q_out[(size_t)i * qd + h * hd + d + half] = (bb * c.x + a * c.y) * qscale;
+    }
+    if (!full) {
+        const size_t trow = (size_t)slab_off[b] + T;
+        for (int p = threadIdx.x; p < Hkv * half; p += blockDim.x) {
+            const int h = p / half, d = p - h * half;
+            const float2 c = csb[d];
+            const float a = row[qd + h * hd + d], bb = row[qd + h * hd + d + half];
+            KT* dst = kc + ((size_t)h * cap_total + trow) * hd;
+            dst[d] = from_f32<KT>(a * c.x - bb * c.y);
+            dst[d + half] = from_f32<KT>(bb * c.x + a * c.y);
+        }
+        for (int p = threadIdx.x; p < kvd; p += blockDim.x) {
+            const int h = p / hd, d = p - h * hd;
+            vc[((size_t)h * cap_total + trow) * hd + d] = from_f32<KT>(row[qd + kvd + p]);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (full) atomicOr(flags, FIRST_FLAG_KV_FULL);
+        else len_l[b] = T + 1;
+    }
+}
+
+// act[i][f] = silu(gate) * up from gu[i] = [gate(F) | up(F)]; optional bf16 hi/lo split.
+__global__ void __launch_bounds__(256) silu_mul(const float* __restrict__ gu, int m, int F, float* __restrict__ act,
+                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    const size_t n = (size_t)m * F;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        const size_t i = e / F, f = e - i * F;
+        const float g = gu[i * 2 * F + f], u = gu[i * 2 * F + F + f];
+        const float y = g / (1.f + expf(-g)) * u;
+        if (act) act[e] = y;
+        if (hi) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            hi[e] = h;
+            lo[e] = __float2bfloat16_rn(y - __bfloat162float(h));
+        }
+    }
+}
+
+// End of a step: greedy next token per row (lowest index among equal maxima) and pos += 1.
+__global__ void __launch_bounds__(256) step_end(const float* __restrict__ logits, int V, int32_t* __restrict__ next,
+                                                int32_t* __restrict__ pos) {
+    const int b = blockIdx.x;
+    if (next && logits) {
+        __shared__ float bv[256];
+        __shared__ int bi[256];
+        const float* row = logits + (size_t)b * V;
+        float best = -INFINITY;
+        int besti = 0x7fffffff;
+        for (int i = threadIdx.x; i < V; i += 256) {
+            const float v = row[i];
+            if (v > best || (v == best && i < besti)) { best = v; besti = i; }
+        }
+        bv[threadIdx.x] = best;
+        bi[threadIdx.x] = besti;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (threadIdx.x < o) {
+                const float v = bv[threadIdx.x + o];
+                const int j = bi[threadIdx.x + o];
+                if (v > bv[threadIdx.x] || (v == bv[threadIdx.x] && j < bi[threadIdx.x])) {
+                    bv[threadIdx.x] = v;
+                    bi[threadIdx.x] = j;
+                }
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) next[b] = bi[0] == 0x7fffffff ? 0 : bi[0];
+    }
+    if (threadIdx.x == 0) pos[b] += 1;
+}
+
+}  // namespace first
