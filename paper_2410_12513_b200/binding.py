@@ -1,0 +1,239 @@
+"""ctypes binding of ``libfirst.so``: the same calls as ``include/first.h``, taking torch
+CUDA tensors.  Argument marshalling only -- no arithmetic happens here."""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIBPATH = _PKG / "libfirst.so"
+_lib = None
+
+FIRST_DTYPE_F32, FIRST_DTYPE_BF16 = 0, 1
+MEAN_OF_SIGMOID, SIGMOID_OF_MEAN = 0, 1
+FLAG_KV_FULL, FLAG_BAD_TOKEN, FLAG_BAD_MASK, FLAG_WAIT_EXPIRED, FLAG_EMPTY_SEQ = 1, 2, 4, 8, 16
+
+
+class FirstError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        msg = lib().first_status_string(status).decode()
+        super().__init__(f"{what}: status {status} ({msg})")
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "ffn_dim",
+                                         "vocab")] + \
+               [("rope_base", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32), ("max_batch", C.c_int32),
+                ("max_tokens_per_seq", C.c_int32)]
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("attn_norm", C.POINTER(C.c_void_p)), ("wqkv", C.POINTER(C.c_void_p)),
+                ("wo", C.POINTER(C.c_void_p)), ("ffn_norm", C.POINTER(C.c_void_p)),
+                ("w_gate_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+
+
+class KVCacheC(C.Structure):
+    _fields_ = [("k", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)), ("slab_off", C.c_void_p),
+                ("slab_cap", C.c_void_p), ("len", C.c_void_p), ("pos", C.c_void_p), ("cap_total", C.c_int64)]
+
+
+def library_path() -> Path:
+    return _LIBPATH
+
+
+def lib():
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not _LIBPATH.exists():
+            raise FileNotFoundError(f"{_LIBPATH} is missing: build it with `python -m paper_2410_12513_b200.build`")
+        L = C.CDLL(str(_LIBPATH))
+        L.first_status_string.restype = C.c_char_p
+        L.first_status_string.argtypes = [C.c_int]
+        L.first_create.argtypes = [C.POINTER(ModelDesc), C.POINTER(Weights), C.POINTER(C.c_void_p)]
+        L.first_destroy.argtypes = [C.c_void_p]
+        L.first_prefill_route.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
+                                          C.c_int64, C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]
+        L.first_set_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.first_get_plan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.first_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(KVCacheC), C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p]
+        L.first_last_device_flags.argtypes = [C.c_void_p, C.POINTER(C.c_uint32), C.c_void_p]
+        L.first_launch_count.restype = C.c_int64
+        L.first_launch_count.argtypes = [C.c_void_p]
+        L.first_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int64]
+        for name in ("first_create", "first_destroy", "first_prefill_route", "first_set_mask", "first_get_plan",
+                     "first_decode_step", "first_last_device_flags", "first_set_option"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _dev(t, dtype=None, what="tensor"):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{what} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{what} must have dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _ptr_array(tensors, dtype, what):
+    arr = (C.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else _dev(t, dtype, f"{what}[{i}]").value
+    return arr
+
+
+class KVCache:
+    """Marshals caller-owned cache tensors into ``first_kv_cache``.
+
+    k, v: lists (one per layer) of CUDA tensors [Hkv][cap_total][hd] (None allowed for
+    layers no sequence keeps); slab_off int64 [B]; slab_cap int32 [B]; len int32 [L][B];
+    pos int32 [B]."""
+
+    def __init__(self, k, v, slab_off, slab_cap, len_, pos):
+        self.k, self.v, self.slab_off, self.slab_cap, self.len, self.pos = k, v, slab_off, slab_cap, len_, pos
+        first = next(t for t in k if t is not None)
+        self._ka = _ptr_array(k, first.dtype, "kv.k")
+        self._va = _ptr_array(v, first.dtype, "kv.v")
+        self.c = KVCacheC(C.cast(self._ka, C.POINTER(C.c_void_p)), C.cast(self._va, C.POINTER(C.c_void_p)),
+                          _dev(slab_off, torch.int64, "slab_off"), _dev(slab_cap, torch.int32, "slab_cap"),
+                          _dev(len_, torch.int32, "len"), _dev(pos, torch.int32, "pos"), int(first.shape[1]))
+
+
+def first_create(shape, dtype, max_batch, max_tokens_per_seq, weights):
+    """weights: dict with embed, lm_head, final_norm and per-layer lists attn_norm, wqkv, wo,
+    ffn_norm, w_gate_up, w_down (CUDA tensors).  Returns (handle, keepalive)."""
+    wd = torch.float32 if dtype == FIRST_DTYPE_F32 else torch.bfloat16
+    desc = ModelDesc(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                     shape.ffn_dim, shape.vocab, float(shape.rope_base), float(shape.rms_eps), dtype,
+                     int(max_batch), int(max_tokens_per_seq))
+    arrs = {k: _ptr_array(weights[k], torch.float32 if k.endswith("norm") else wd, k)
+            for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")}
+    w = Weights(_dev(weights["embed"], wd, "embed"), _dev(weights["lm_head"], wd, "lm_head"),
+                _dev(weights["final_norm"], torch.float32, "final_norm"),
+                *[C.cast(arrs[k], C.POINTER(C.c_void_p)) for k in
+                  ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")])
+    h = C.c_void_p()
+    rc = lib().first_create(C.byref(desc), C.byref(w), C.byref(h))
+    if rc:
+        raise FirstError(rc, "first_create")
+    return h, (weights, arrs)
+
+
+def first_destroy(h):
+    lib().first_destroy(h)
+
+
+def first_prefill_route(h, layer, hidden, cu_seqlens, router_w, router_b, tau, mode, mask, scores=None,
+                        stream=None):
+    if hidden.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("hidden must be float32 or bfloat16")
+    hd = FIRST_DTYPE_F32 if hidden.dtype == torch.float32 else FIRST_DTYPE_BF16
+    rc = lib().first_prefill_route(h, layer, _dev(hidden, None, "hidden"), hd,
+                                   _dev(cu_seqlens, torch.int32, "cu_seqlens"), cu_seqlens.numel() - 1,
+                                   hidden.shape[0], _dev(router_w, torch.float32, "router_w"),
+                                   _dev(router_b, torch.float32, "router_b"), float(tau), int(mode),
+                                   _dev(mask, torch.uint8, "mask"), _dev(scores, torch.float32, "scores"),
+                                   _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_prefill_route")
+
+
+def first_set_mask(h, mask, stream=None):
+    rc = lib().first_set_mask(h, _dev(mask, torch.uint8, "mask"), mask.shape[0], _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_set_mask")
+
+
+def first_get_plan(h, B, L):
+    import numpy as np
+    idx = np.empty((L, B), dtype=np.int32)
+    cnt = np.empty((L,), dtype=np.int32)
+    slot = np.empty((L, B), dtype=np.int32)
+    rc = lib().first_get_plan(h, idx.ctypes.data, cnt.ctypes.data, slot.ctypes.data)
+    if rc:
+        raise FirstError(rc, "first_get_plan")
+    return idx, cnt, slot
+
+
+def first_decode_step(h, tokens, kv: KVCache, logits=None, next_tokens=None, layer_inputs=None, stream=None):
+    rc = lib().first_decode_step(h, _dev(tokens, torch.int32, "tokens"), C.byref(kv.c),
+                                 _dev(logits, torch.float32, "logits"),
+                                 _dev(next_tokens, torch.int32, "next_tokens"),
+                                 _dev(layer_inputs, torch.float32, "layer_inputs"), _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_decode_step")
+
+
+def first_last_device_flags(h, stream=None):
+    fl = C.c_uint32(0)
+    rc = lib().first_last_device_flags(h, C.byref(fl), _stream(stream))
+    if rc not in (0, -6):
+        raise FirstError(rc, "first_last_device_flags")
+    return fl.value
+
+
+def first_set_option(h, name, value):
+    rc = lib().first_set_option(h, name.encode(), int(value))
+    if rc:
+        raise FirstError(rc, "first_set_option")
+
+
+class FirstContext:
+    """Owns one library context; methods mirror the C calls."""
+
+    def __init__(self, shape, dtype, max_batch, max_tokens_per_seq, weights):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required; there is no CPU path")
+        self.shape, self.dtype = shape, dtype
+        self.h, self._keep = first_create(shape, dtype, max_batch, max_tokens_per_seq, weights)
+
+    def close(self):
+        if self.h is not None:
+            first_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def prefill_route(self, layer, hidden, cu_seqlens, router_w, router_b, tau, mode, mask, scores=None, stream=None):
+        first_prefill_route(self.h, layer, hidden, cu_seqlens, router_w, router_b, tau, mode, mask, scores, stream)
+
+    def set_mask(self, mask, stream=None):
+        first_set_mask(self.h, mask, stream)
+        self.B = mask.shape[0]
+
+    def get_plan(self):
+        return first_get_plan(self.h, self.B, self.shape.n_layers)
+
+    def decode_step(self, tokens, kv, logits=None, next_tokens=None, layer_inputs=None, stream=None):
+        first_decode_step(self.h, tokens, kv, logits, next_tokens, layer_inputs, stream)
+
+    def device_flags(self, stream=None):
+        return first_last_device_flags(self.h, stream)
+
+    def launch_count(self):
+        return int(lib().first_launch_count(self.h))
+
+    def set_option(self, name, value):
+        first_set_option(self.h, name, value)

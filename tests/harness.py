@@ -1,0 +1,148 @@
+"""Test-side glue: the same seeded inputs laid out for the host oracle (numpy) and for the
+CUDA library (torch), router-weight calibration against the oracle, and comparisons."""
+from __future__ import annotations
+
+import numpy as np
+
+import first_inputs as fi
+import oracle
+
+
+# ------------------------------------------------------------------ oracle side
+def oracle_model(shape, weights):
+    return oracle.OracleModel(oracle.Shape(**shape.asdict()), weights)
+
+
+def widen(a):
+    return fi.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a
+
+
+# ------------------------------------------------------------------ CUDA side
+def to_dev(a, bf16):
+    import torch
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t
+
+
+def gpu_weights(w, layers=None):
+    """Generator dict -> the layout first_create takes (q,k,v rows concatenated; gate,up rows
+    concatenated).  Layers not materialised stay None."""
+    import torch
+    L = len(w["wq"])
+    bf16 = w["embed"].dtype == np.uint16
+    out = {"embed": to_dev(w["embed"], bf16), "lm_head": to_dev(w["lm_head"], bf16),
+           "final_norm": to_dev(w["final_norm"], False)}
+    for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
+        out[k] = [None] * L
+    for l in range(L):
+        if w["wq"][l] is None:
+            continue
+        out["attn_norm"][l] = to_dev(w["attn_norm"][l], False)
+        out["ffn_norm"][l] = to_dev(w["ffn_norm"][l], False)
+        out["wqkv"][l] = torch.cat([to_dev(w[k][l], bf16) for k in ("wq", "wk", "wv")], 0).contiguous()
+        out["wo"][l] = to_dev(w["wo"][l], bf16)
+        out["w_gate_up"][l] = torch.cat([to_dev(w[k][l], bf16) for k in ("wg", "wu")], 0).contiguous()
+        out["w_down"][l] = to_dev(w["wd"][l], bf16)
+    return out
+
+
+class GpuKV:
+    """Caller-owned cache tensors in the library's layout, plus the binding struct."""
+
+    def __init__(self, shape, caps, bf16, layers=None):
+        import torch
+        from paper_2410_12513_b200 import KVCache
+        caps = np.asarray(caps, dtype=np.int32)
+        self.shape, self.B, self.L = shape, len(caps), shape.n_layers
+        self.caps = caps
+        self.off = np.concatenate([[0], np.cumsum(caps[:-1], dtype=np.int64)]).astype(np.int64)
+        tot = int(caps.sum())
+        dt = torch.bfloat16 if bf16 else torch.float32
+        layers = range(self.L) if layers is None else layers
+        self.k = [None] * self.L
+        self.v = [None] * self.L
+        for l in layers:
+            self.k[l] = torch.zeros((shape.n_kv_heads, tot, shape.head_dim), dtype=dt, device="cuda")
+            self.v[l] = torch.zeros((shape.n_kv_heads, tot, shape.head_dim), dtype=dt, device="cuda")
+        self.slab_off = torch.from_numpy(self.off).cuda()
+        self.slab_cap = torch.from_numpy(caps).cuda()
+        self.len = torch.zeros((self.L, self.B), dtype=torch.int32, device="cuda")
+        self.pos = torch.zeros((self.B,), dtype=torch.int32, device="cuda")
+        self.c = KVCache(self.k, self.v, self.slab_off, self.slab_cap, self.len, self.pos)
+
+    def load_rows(self, l, b, k_rows, v_rows):
+        """k_rows/v_rows: numpy [n][Hkv*hd] token-major (float32 or bf16 bits)."""
+        import torch
+        n = k_rows.shape[0]
+        s = self.shape
+        o = int(self.off[b])
+        for dst, src in ((self.k[l], k_rows), (self.v[l], v_rows)):
+            t = to_dev(src, src.dtype == np.uint16).to(dst.dtype)
+            dst[:, o:o + n, :] = t.view(n, s.n_kv_heads, s.head_dim).permute(1, 0, 2)
+
+    def set_len(self, lens, pos):
+        import torch
+        self.len.copy_(torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)))
+        self.pos.copy_(torch.from_numpy(np.ascontiguousarray(pos, dtype=np.int32)))
+
+    def rows_host(self, l, b):
+        """-> (k, v) numpy float32 [cap][Hkv*hd] token-major."""
+        o, cp = int(self.off[b]), int(self.caps[b])
+        f = lambda t: t[:, o:o + cp, :].permute(1, 0, 2).reshape(cp, -1).float().cpu().numpy()
+        return f(self.k[l]), f(self.v[l])
+
+
+def synthetic_caches(shape, lens, caps, seed, bf16, layers=None, with_gpu=True):
+    """Stand-in prefilled caches N(0,1) for every (layer, sequence): identical values on both
+    sides.  lens: [B] tokens present in every layer; pos = lens."""
+    B, L = len(lens), shape.n_layers
+    okv = oracle.OracleKV(oracle.Shape(**shape.asdict()), caps)
+    gkv = GpuKV(shape, caps, bf16, layers) if with_gpu else None
+    layers = range(L) if layers is None else layers
+    for l in layers:
+        for b in range(B):
+            n = int(lens[b])
+            kr = fi.synthetic_kv_rows(n, shape.kv_dim, seed, f"k{l}_{b}", bf16)
+            vr = fi.synthetic_kv_rows(n, shape.kv_dim, seed, f"v{l}_{b}", bf16)
+            ko, vo = okv.rows(l, b)
+            ko[:n] = widen(kr)
+            vo[:n] = widen(vr)
+            if gkv is not None:
+                gkv.load_rows(l, b, kr, vr)
+    okv.len[:] = np.asarray(lens, dtype=np.int32)[None, :]
+    okv.pos[:] = np.asarray(lens, dtype=np.int32)
+    if gkv is not None:
+        gkv.set_len(okv.len, okv.pos)
+    return okv, gkv
+
+
+# ------------------------------------------------------------------ router calibration
+def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3):
+    """Router weights w[D] (no bias) that realise `target_keep` on the given per-sequence hidden
+    states with every oracle score at least `margin` away from tau.  Least-norm solve on the
+    pooled means (B <= D), scaled up until the oracle's own scores clear the margin."""
+    B = len(hiddens)
+    pooled = np.stack([h.astype(np.float64).mean(0) for h in hiddens])  # [B][D]
+    t = np.where(np.asarray(target_keep) > 0, 1.0, -1.0)
+    c = 0.25
+    for _ in range(12):
+        w = (np.linalg.pinv(pooled) @ (c * t)).astype(np.float32)
+        rho = np.array([oracle.route(h, w, None, tau, mode)[0] for h in hiddens])
+        keep = rho >= tau
+        if (keep == (t > 0)).all() and np.abs(rho - tau).min() >= margin:
+            return w, rho
+        c *= 2.0
+    raise AssertionError("router calibration failed")
+
+
+# ------------------------------------------------------------------ comparisons
+def logits_check(got, ref, rel=2e-2):
+    """max-abs error relative to the row's logit range, and argmax agreement per row."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rng = ref.max(-1) - ref.min(-1)
+    err = np.abs(got - ref).max(-1) / rng
+    agree = got.argmax(-1) == ref.argmax(-1)
+    return err, agree
