@@ -185,6 +185,18 @@ int first_last_device_flags(first_ctx *ctx, uint32_t *flags, void *stream);
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t first_launch_count(const first_ctx *ctx);
 
+/* Measurement aid (the paper has no counterpart): per-kernel-class device timing.  While
+ * enabled, every launch of this context is bracketed by a CUDA event pair on its stream
+ * (this serialises launches slightly; leave it off when timing whole steps).
+ * first_profile(ctx, 1) clears the totals and starts; first_profile(ctx, 0) stops.
+ * first_profile_read waits for `stream`, folds the pending event pairs into the totals and
+ * copies them out: ms[k] = total device milliseconds of class k, launches[k] = its launch
+ * count, for k < first_kernel_class_count() (n must be at least that).  Host arrays. */
+int first_profile(first_ctx *ctx, int32_t enable);
+int first_profile_read(first_ctx *ctx, int32_t n, double *ms, int64_t *launches, void *stream);
+int32_t first_kernel_class_count(void);
+const char *first_kernel_class_name(int32_t k);
+
 /* Select kernel paths for A/B measurements.  Names: "max_gemv_rows" = largest active-row
  * count served by the CUDA-core GEMV path (rows above it use the tensor-core path when
  * the dtype is bfloat16); "attn_simple" = 1 forces the general attention kernel.  A

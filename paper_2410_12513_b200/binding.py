@@ -68,6 +68,13 @@ def lib():
         L.first_launch_count.restype = C.c_int64
         L.first_launch_count.argtypes = [C.c_void_p]
         L.first_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int64]
+        L.first_profile.argtypes = [C.c_void_p, C.c_int32]
+        L.first_profile.restype = C.c_int
+        L.first_profile_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.first_profile_read.restype = C.c_int
+        L.first_kernel_class_count.restype = C.c_int32
+        L.first_kernel_class_name.restype = C.c_char_p
+        L.first_kernel_class_name.argtypes = [C.c_int32]
         for name in ("first_create", "first_destroy", "first_prefill_route", "first_set_mask", "first_get_plan",
                      "first_decode_step", "first_last_device_flags", "first_set_option"):
             getattr(L, name).restype = C.c_int
@@ -196,6 +203,23 @@ def first_set_option(h, name, value):
         raise FirstError(rc, "first_set_option")
 
 
+def first_profile(h, enable):
+    rc = lib().first_profile(h, int(bool(enable)))
+    if rc:
+        raise FirstError(rc, "first_profile")
+
+
+def first_profile_read(h, stream=None):
+    """-> {kernel class name: (total device ms, launches)}"""
+    n = lib().first_kernel_class_count()
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    rc = lib().first_profile_read(h, n, ms, cnt, _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_profile_read")
+    return {lib().first_kernel_class_name(k).decode(): (ms[k], cnt[k]) for k in range(n)}
+
+
 class FirstContext:
     """Owns one library context; methods mirror the C calls."""
 
@@ -237,3 +261,9 @@ class FirstContext:
 
     def set_option(self, name, value):
         first_set_option(self.h, name, value)
+
+    def profile(self, enable):
+        first_profile(self.h, enable)
+
+    def profile_read(self, stream=None):
+        return first_profile_read(self.h, stream)

@@ -25,6 +25,13 @@ using namespace first;
 
 static thread_local char g_last_cuda_error[256] = "";
 
+enum KernelClass { kClsStepBegin = 0, kClsRmsnorm, kClsGemv, kClsGemmTc, kClsRopeAppend, kClsAttn, kClsAttnCombine,
+                   kClsSiluMul, kClsStepEnd, kClsRouterScores, kClsRouterFinalize, kClsPlan, kNumClasses };
+static const char* const kClassNames[kNumClasses] = {"step_begin", "rmsnorm_rows", "gemv_rows", "gemm_tc",
+                                                     "rope_append", "attn_split", "attn_combine", "silu_mul",
+                                                     "step_end", "router_token_scores", "router_finalize",
+                                                     "plan_compact"};
+
 struct first_ctx {
     first_model_desc d{};
     const void *embed = nullptr, *lm_head = nullptr;
@@ -47,6 +54,12 @@ struct first_ctx {
     int B = 0;
     bool has_mask = false;
     int64_t launches = 0;
+    // per-kernel-class timing (off unless first_profile enables it)
+    bool profiling = false;
+    std::vector<cudaEvent_t> ev_pool;
+    std::vector<int> ev_cls;  // class of event pair i (events 2i, 2i+1)
+    double prof_ms[kNumClasses] = {};
+    int64_t prof_launches[kNumClasses] = {};
     // options
     int max_gemv_rows = -1;
     int attn_simple = -1;
@@ -60,8 +73,36 @@ int dev_alloc(T** p, size_t n) {
     return FIRST_OK;
 }
 
-int check_launch(first_ctx* c, int n = 1) {
-    c->launches += n;
+// Brackets one kernel launch: counts it and, when profiling, records an event pair around it.
+struct Launch {
+    first_ctx* c;
+    cudaStream_t st;
+    bool on;
+    Launch(first_ctx* c_, cudaStream_t st_, int cls) : c(c_), st(st_), on(c_->profiling) {
+        c->launches += 1;
+        if (on) {
+            const size_t i = c->ev_cls.size();
+            while (c->ev_pool.size() < 2 * (i + 1)) {
+                cudaEvent_t e;
+                if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+                c->ev_pool.push_back(e);
+            }
+            c->ev_cls.push_back(cls);
+            cudaEventRecord(c->ev_pool[2 * i], st);
+        }
+    }
+    ~Launch() {
+        if (on) cudaEventRecord(c->ev_pool[2 * (c->ev_cls.size() - 1) + 1], st);
+    }
+};
+
+#define FIRST_LAUNCH(cls, ...)      \
+    do {                            \
+        Launch guard_(c, st, cls);  \
+        __VA_ARGS__;                \
+    } while (0)
+
+int check_launch(first_ctx*) {
     CU_TRY(cudaGetLastError());
     return FIRST_OK;
 }
@@ -73,10 +114,10 @@ int launch_gemv(first_ctx* c, cudaStream_t st, const void* W, int n_out, int K, 
     for (int r0 = 0; r0 < m; r0 += 8) {
         const int rv = std::min(8, m - r0);
         const WT* w = static_cast<const WT*>(W);
-        if (rv == 1) gemv_rows<WT, 1, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx);
-        else if (rv == 2) gemv_rows<WT, 2, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx);
-        else if (rv <= 4) gemv_rows<WT, 4, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx);
-        else gemv_rows<WT, 8, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx);
+        if (rv == 1) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 1, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
+        else if (rv == 2) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 2, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
+        else if (rv <= 4) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 4, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
+        else FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 8, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
         int rc = check_launch(c);
         if (rc) return rc;
     }
@@ -89,8 +130,9 @@ int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* 
     dim3 grid(S, c->d.n_kv_heads, m);
 #define FIRST_ATTN_CASE(G)                                                                                   \
     case G:                                                                                                  \
-        attn_split_simple<KT, HD, G><<<grid, 128, 0, st>>>(c->q, kc, vc, kv->cap_total, kv->slab_off, len_l, \
-                                                           idx, c->d.n_q_heads, c->o_part, c->ml_part);     \
+        FIRST_LAUNCH(kClsAttn, (attn_split_simple<KT, HD, G><<<grid, 128, 0, st>>>(                          \
+                                   c->q, kc, vc, kv->cap_total, kv->slab_off, len_l, idx, c->d.n_q_heads,    \
+                                   c->o_part, c->ml_part)));                                                 \
         break;
     switch (c->group) {
         FIRST_ATTN_CASE(1)
@@ -122,8 +164,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const first_model_desc& d = c->d;
     const int B = c->B, D = d.d_model, F = d.ffn_dim, V = d.vocab, L = d.n_layers, hd = d.head_dim;
     int rc;
-    step_begin<WT><<<B, 256, 0, st>>>(tokens, static_cast<const WT*>(c->embed), D, V, kv->pos, c->inv_freq, hd / 2,
-                                      c->x, c->cs, c->flags);
+    FIRST_LAUNCH(kClsStepBegin, (step_begin<WT><<<B, 256, 0, st>>>(tokens, static_cast<const WT*>(c->embed), D, V, kv->pos, c->inv_freq, hd / 2,
+                                      c->x, c->cs, c->flags)));
     if ((rc = check_launch(c))) return rc;
 
     int S = (d.max_tokens_per_seq + 255) / 256;
@@ -139,22 +181,22 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const int32_t* idx = c->idx + (size_t)l * B;
         int32_t* len_l = kv->len + (size_t)l * B;
         // attention half
-        rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->attn_norm[l], d.rms_eps, c->xn, nullptr, nullptr);
+        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->attn_norm[l], d.rms_eps, c->xn, nullptr, nullptr)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_gemv<WT, kStore>(c, st, c->wqkv[l], c->qkvd, D, c->xn, m, c->qkv, c->qkvd, nullptr))) return rc;
-        rope_append<WT><<<m, 256, 0, st>>>(c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
+        FIRST_LAUNCH(kClsRopeAppend, (rope_append<WT><<<m, 256, 0, st>>>(c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total,
-                                           kv->slab_off, kv->slab_cap, len_l, c->flags);
+                                           kv->slab_off, kv->slab_cap, len_l, c->flags)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
-        attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd, c->att, nullptr, nullptr);
+        FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd, c->att, nullptr, nullptr)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_gemv<WT, kScatterAdd>(c, st, c->wo[l], D, c->qd, c->att, m, c->x, D, idx))) return rc;
         // feed-forward half
-        rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->ffn_norm[l], d.rms_eps, c->xn, nullptr, nullptr);
+        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->ffn_norm[l], d.rms_eps, c->xn, nullptr, nullptr)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_gemv<WT, kStore>(c, st, c->w_gate_up[l], 2 * F, D, c->xn, m, c->gu, 2 * F, nullptr))) return rc;
-        silu_mul<<<std::min((m * F + 255) / 256, c->n_sm * 8), 256, 0, st>>>(c->gu, m, F, c->act, nullptr, nullptr);
+        FIRST_LAUNCH(kClsSiluMul, (silu_mul<<<std::min((m * F + 255) / 256, c->n_sm * 8), 256, 0, st>>>(c->gu, m, F, c->act, nullptr, nullptr)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_gemv<WT, kScatterAdd>(c, st, c->w_down[l], D, F, c->act, m, c->x, D, idx))) return rc;
     }
@@ -164,11 +206,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         lg = c->logits_int;
     }
     if (lg) {
-        rmsnorm_rows<<<B, 256, 0, st>>>(c->x, nullptr, D, c->final_norm, d.rms_eps, c->xn, nullptr, nullptr);
+        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<B, 256, 0, st>>>(c->x, nullptr, D, c->final_norm, d.rms_eps, c->xn, nullptr, nullptr)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_gemv<WT, kStore>(c, st, c->lm_head, V, D, c->xn, B, lg, V, nullptr))) return rc;
     }
-    step_end<<<B, 256, 0, st>>>(lg, V, next_tokens, kv->pos);
+    FIRST_LAUNCH(kClsStepEnd, (step_end<<<B, 256, 0, st>>>(lg, V, next_tokens, kv->pos)));
     return check_launch(c);
 }
 
@@ -262,6 +304,7 @@ int first_destroy(first_ctx* c) {
                     c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     delete c;
     return FIRST_OK;
 }
@@ -281,16 +324,16 @@ int first_prefill_route(first_ctx* c, int32_t layer, const void* hidden, int32_t
     const int blocks = (int)std::min<int64_t>(want, (int64_t)c->n_sm * 8);
     const size_t smem = (size_t)D * sizeof(float);
     if (hidden_dtype == FIRST_DTYPE_BF16)
-        router_token_scores<__nv_bfloat16><<<blocks, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(hidden),
+        FIRST_LAUNCH(kClsRouterScores, (router_token_scores<__nv_bfloat16><<<blocks, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(hidden),
                                                                       total_tokens, D, router_w, router_b, mode,
-                                                                      c->tokscore);
+                                                                      c->tokscore)));
     else
-        router_token_scores<float><<<blocks, 256, smem, st>>>(static_cast<const float*>(hidden), total_tokens, D,
-                                                              router_w, router_b, mode, c->tokscore);
+        FIRST_LAUNCH(kClsRouterScores, (router_token_scores<float><<<blocks, 256, smem, st>>>(static_cast<const float*>(hidden), total_tokens, D,
+                                                              router_w, router_b, mode, c->tokscore)));
     int rc = check_launch(c);
     if (rc) return rc;
-    router_finalize<<<B, 256, 0, st>>>(c->tokscore, cu_seqlens, c->d.n_layers, layer, mode, tau, mask, scores,
-                                       c->flags);
+    FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->tokscore, cu_seqlens, c->d.n_layers, layer, mode, tau, mask, scores,
+                                       c->flags)));
     return check_launch(c);
 }
 
@@ -299,7 +342,7 @@ int first_set_mask(first_ctx* c, const uint8_t* mask, int32_t B, void* stream) {
     if (B > c->d.max_batch) return FIRST_E_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c->has_mask = false;
-    plan_compact<<<c->d.n_layers, 32, 0, st>>>(mask, B, c->d.n_layers, c->idx, c->cnt, c->slot, c->flags);
+    FIRST_LAUNCH(kClsPlan, (plan_compact<<<c->d.n_layers, 32, 0, st>>>(mask, B, c->d.n_layers, c->idx, c->cnt, c->slot, c->flags)));
     int rc = check_launch(c);
     if (rc) return rc;
     uint32_t fl = 0;
@@ -346,6 +389,34 @@ int first_last_device_flags(first_ctx* c, uint32_t* flags, void* stream) {
 }
 
 int64_t first_launch_count(const first_ctx* c) { return c ? c->launches : 0; }
+
+int first_profile(first_ctx* c, int32_t enable) {
+    if (!c) return FIRST_E_ARG;
+    c->profiling = enable != 0;
+    c->ev_cls.clear();
+    for (int k = 0; k < kNumClasses; ++k) { c->prof_ms[k] = 0.0; c->prof_launches[k] = 0; }
+    return FIRST_OK;
+}
+
+int first_profile_read(first_ctx* c, int32_t n, double* ms, int64_t* launches, void* stream) {
+    if (!c || !ms || !launches || n < kNumClasses) return FIRST_E_ARG;
+    CU_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    for (size_t i = 0; i < c->ev_cls.size(); ++i) {
+        float t = 0.f;
+        CU_TRY(cudaEventElapsedTime(&t, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+        c->prof_ms[c->ev_cls[i]] += t;
+        c->prof_launches[c->ev_cls[i]] += 1;
+    }
+    c->ev_cls.clear();
+    for (int k = 0; k < n; ++k) {
+        ms[k] = k < kNumClasses ? c->prof_ms[k] : 0.0;
+        launches[k] = k < kNumClasses ? c->prof_launches[k] : 0;
+    }
+    return FIRST_OK;
+}
+
+int32_t first_kernel_class_count(void) { return kNumClasses; }
+const char* first_kernel_class_name(int32_t k) { return (k >= 0 && k < kNumClasses) ? kClassNames[k] : ""; }
 
 int first_set_option(first_ctx* c, const char* name, int64_t value) {
     if (!c || !name) return FIRST_E_ARG;
