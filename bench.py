@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the router-selective decode step (decode tokens/s and step latency at the
+Llama-3-8B shape, with the achieved fraction of the HBM roofline).
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the host oracle, bounded sample
+
+One step = one routed decode step of the whole batch (embedding, every layer for the rows
+that keep it, final norm, lm_head, greedy token).  Routing and the per-layer row plan are
+done once per batch, before the timed steps, and reported separately.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import first_inputs as fi  # noqa: E402
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+
+WORKLOADS = {
+    # name: (shape, B, prompt lo, prompt hi, default steps, mask recipe)
+    "cfg1_1b_b1": dict(shape="1b", B=1, lo=512, hi=512, steps=256, mask=("fraction", 0.25, 0.25)),
+    "cfg2_8b_b32": dict(shape="8b", B=32, lo=128, hi=2048, steps=128, mask=("fraction", 0.10, 0.40)),
+    "cfg3_8b_b256": dict(shape="8b", B=256, lo=1024, hi=4096, steps=64, mask=("bernoulli", 0.7)),
+    "cfg4_8b_b64": dict(shape="8b", B=64, lo=1024, hi=1024, steps=128, mask=("aligned", 0.25)),
+}
+SHAPES = {"1b": fi.LLAMA_1B, "8b": fi.LLAMA_8B, "3b": fi.LLAMA_3B}
+
+
+def make_mask(recipe, B, L, seed):
+    kind = recipe[0]
+    if kind == "fraction":
+        return fi.mask_skip_fraction(B, L, recipe[1], recipe[2], seed)
+    if kind == "bernoulli":
+        return fi.mask_bernoulli(B, L, recipe[1], seed)
+    if kind == "aligned":
+        return fi.mask_aligned(B, L, recipe[1])
+    if kind == "independent":
+        return fi.mask_independent(B, L, recipe[1], seed)
+    if kind == "dense":
+        return np.ones((B, L), np.uint8)
+    raise ValueError(kind)
+
+
+def byte_model(shape, mask, lens, kv_elem=2, w_elem=2):
+    """Roofline bytes of one step: weights of layers with any active row + KV of active rows
+    (strict), and the same plus lm_head, embedding rows, KV appends and the logits (full)."""
+    B, L = mask.shape
+    cnt = mask.sum(0)
+    w_layer = shape.layer_params() * w_elem
+    kv_tok = 2 * shape.kv_dim * kv_elem
+    weights = int((cnt > 0).sum()) * w_layer
+    kv = int(sum(kv_tok * (int(lens[b]) + 1) for b in range(B) for l in range(L) if mask[b, l]))
+    strict = weights + kv
+    full = strict + shape.vocab * shape.d_model * w_elem + B * shape.d_model * w_elem + int(cnt.sum()) * kv_tok \
+        + B * shape.vocab * 4
+    return dict(strict=strict, full=full, weights=weights, kv=kv, lm_head=shape.vocab * shape.d_model * w_elem)
+
+
+class ClockSampler:
+    """nvidia-smi sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.25)
+            self.proc.terminate()
+            self.t.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- oracle arm
+def oracle_sample(shape, mask, lens, seed, rows=4, layers=2):
+    """Time the host oracle on a bounded sample of the workload: `rows` sequences of the batch
+    (their real cache lengths, stand-in cache contents), `layers` decoder layers of the same
+    width, plus final norm + lm_head; extrapolate to the whole step by the mask's kept
+    (row, layer) count."""
+    sys.path.insert(0, str(ROOT / "tests"))
+    import oracle
+    from harness import oracle_model, synthetic_caches
+    B, L = mask.shape
+    rows = min(rows, B)
+    sub = fi.ModelShape(layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn_dim,
+                        shape.vocab, shape.rope_base, shape.rms_eps)
+    w = fi.make_weights(sub, seed, True)
+    om = oracle_model(sub, w)
+    sel = np.linspace(0, B - 1, rows).astype(int)
+    l_sel = [int(lens[b]) for b in sel]
+    okv, _ = synthetic_caches(sub, l_sel, [n + 2 for n in l_sel], seed, True, with_gpu=False)
+    toks = fi.tokens(sub, rows, seed, "oracle_tokens")
+    t0 = time.perf_counter()
+    oracle.decode_step(om, toks, np.zeros((rows, layers), np.uint8), okv)
+    t_head = (time.perf_counter() - t0) / rows
+    t0 = time.perf_counter()
+    oracle.decode_step(om, toks, np.ones((rows, layers), np.uint8), okv)
+    t_all = time.perf_counter() - t0
+    t_layer = max(t_all - t_head * rows, 0.0) / (rows * layers)
+    kept = int(mask.sum())
+    step_s = kept * t_layer + B * t_head
+    cores = len(os.sched_getaffinity(0))
+    return dict(value=B / step_s, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{rows} of {B} sequences x {layers} of {L} layers + lm_head, 1 step, bf16-valued weights; "
+                       f"{t_layer * 1e3:.1f} ms per (sequence, kept layer), {t_head * 1e3:.1f} ms per sequence for "
+                       f"norm+lm_head; extrapolated to {kept} kept (sequence, layer) pairs",
+                ms_per_step=step_s * 1e3)
+
+
+def run_reference(args, wl, shape, mask, lens):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(shape, mask, lens, 100 + i, rows=2, layers=1)
+        if i >= args.warmup:
+            vals.append(r)
+    ms = float(np.mean([v["ms_per_step"] for v in vals]))
+    value = mask.shape[0] / (ms / 1e3)
+    cb = dict(vals[-1])
+    cb["value"] = value
+    cb.pop("ms_per_step")
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": args.workload, "note": "host oracle on a bounded sample, extrapolated"},
+           "cpu_baseline": cb,
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def run_cuda(args, wl, shape, mask, lens):
+    import torch
+    from paper_2410_12513_b200 import FirstContext, KVCache
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    B, L, K, W = mask.shape[0], shape.n_layers, args.steps, args.warmup
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234 + rank)
+
+    def rnd(shp, std):
+        t = torch.empty(shp, dtype=torch.bfloat16, device=dev)
+        t.normal_(0.0, std, generator=g)
+        return t
+
+    s = shape
+    weights = {"embed": rnd((s.vocab, s.d_model), 0.02), "lm_head": rnd((s.vocab, s.d_model), 0.02),
+               "final_norm": torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g)}
+    for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
+        weights[k] = []
+    for l in range(L):
+        weights["attn_norm"].append(torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g))
+        weights["ffn_norm"].append(torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g))
+        weights["wqkv"].append(rnd((s.q_dim + 2 * s.kv_dim, s.d_model), 0.02))
+        weights["wo"].append(rnd((s.d_model, s.q_dim), 0.02))
+        weights["w_gate_up"].append(rnd((2 * s.ffn_dim, s.d_model), 0.02))
+        weights["w_down"].append(rnd((s.d_model, s.ffn_dim), 0.02))
+
+    phase_steps = W + K
+    caps = (lens + phase_steps + 1).astype(np.int32)
+    off = np.concatenate([[0], np.cumsum(caps[:-1], dtype=np.int64)]).astype(np.int64)
+    tot = int(caps.sum())
+    kk = [rnd((s.n_kv_heads, tot, s.head_dim), 1.0) for _ in range(L)]
+    vv = [rnd((s.n_kv_heads, tot, s.head_dim), 1.0) for _ in range(L)]
+    len0 = torch.from_numpy(np.broadcast_to(lens.astype(np.int32), (L, B)).copy()).to(dev)
+    pos0 = torch.from_numpy(lens.astype(np.int32)).to(dev)
+    len_t, pos_t = len0.clone(), pos0.clone()
+    kv = KVCache(kk, vv, torch.from_numpy(off).to(dev), torch.from_numpy(caps).to(dev), len_t, pos_t)
+    ctx = FirstContext(shape, 1, B, int(caps.max()), weights)
+    stream = torch.cuda.current_stream()
+
+    tok0 = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).to(dev)
+    tok_a, tok_b = tok0.clone(), tok0.clone()
+    mask_t = torch.from_numpy(mask).to(dev)
+    dense_t = torch.ones_like(mask_t)
+
+    def reset():
+        len_t.copy_(len0)
+        pos_t.copy_(pos0)
+        tok_a.copy_(tok0)
+
+    def steps(n):
+        a, b = tok_a, tok_b
+        for _ in range(n):
+            ctx.decode_step(a, kv, None, b)
+            a, b = b, a
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(mask_dev):
+        ctx.set_mask(mask_dev)
+        reset()
+        steps(W)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = ctx.launch_count()
+        e0.record(stream)
+        steps(K)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        launches = ctx.launch_count() - l0
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, launches
+
+    # ---- routing + plan, once per batch (reported, not part of the step)
+    route = None
+    if rank == 0 and not args.no_route:
+        n_tok = int(lens.sum())
+        hid = rnd((n_tok, s.d_model), 1.0)
+        cu = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).to(dev)
+        rw = 0.02 * torch.randn(s.d_model, device=dev, generator=g)
+        rmask = torch.zeros((B, L), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            ctx.prefill_route(0, hid, cu, rw, None, 0.5, 1, rmask)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        reps = 10
+        for i in range(reps):
+            ctx.prefill_route(i % L, hid, cu, rw, None, 0.5, 1, rmask)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        rms = e0.elapsed_time(e1) / reps
+        route = {"ms_per_layer": rms, "hidden_bytes": n_tok * s.d_model * 2,
+                 "GBps": n_tok * s.d_model * 2 / rms / 1e6, "tokens": n_tok}
+        del hid
+
+    sampler = ClockSampler(local)
+    with sampler:
+        ms_total, launches = timed(mask_t)
+    clocks = sampler.summary()
+    ms_step = ms_total / K
+    value = world * B * K / (ms_total / 1e3)
+
+    dense_ms, _ = timed(dense_t)
+    dense_ms /= K
+
+    # ---- end to end through the public call with host buffers
+    ctx.set_mask(mask_t)
+    reset()
+    h_tok = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).pin_memory()
+    h_next = torch.empty(B, dtype=torch.int32).pin_memory()
+
+    def e2e_steps(n):
+        for _ in range(n):
+            tok_a.copy_(h_tok, non_blocking=True)
+            ctx.decode_step(tok_a, kv, None, tok_b)
+            h_next.copy_(tok_b, non_blocking=True)
+            stream.synchronize()
+            h_tok.copy_(h_next)
+
+    e2e_steps(W)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    e2e_steps(K)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": world * B * K / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": B * 4,
+           "d2h_bytes_per_step": B * 4, "ms_per_step": e2e_ms / K}
+
+    # ---- per-kernel-class device time (separate pass: event pairs around every launch)
+    reset()
+    steps(2)
+    torch.cuda.synchronize()
+    kp = min(K, 16)
+    ctx.profile(True)
+    steps(kp)
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    flags = ctx.device_flags()
+    if flags:
+        raise RuntimeError(f"device flags set during the benchmark: {flags}")
+    if rank != 0:
+        return
+
+    mid_lens = lens + W + K // 2
+    bm = byte_model(shape, mask, mid_lens)
+    bm_dense = byte_model(shape, np.ones_like(mask), mid_lens)
+    peaks = {}
+    try:
+        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
+    except Exception:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
+    cls_ms = {k: v[0] / kp for k, v in prof.items() if v[1]}
+    tot_cls = sum(cls_ms.values())
+    cnt = mask.sum(0)
+    proj_bytes = bm["weights"] + bm["lm_head"]
+    alg = {"gemv_rows": proj_bytes, "gemm_tc": proj_bytes, "attn_split": bm["kv"]}
+    if cls_ms.get("gemv_rows") and cls_ms.get("gemm_tc"):
+        alg = {"attn_split": bm["kv"]}  # projections split over two classes: attribute by class below
+    dom = max(cls_ms, key=cls_ms.get)
+    roof = {"bound": "hbm", "kernel": dom, "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "traffic": None,
+            "ms_per_step": cls_ms[dom], "share_of_kernel_time": cls_ms[dom] / tot_cls}
+    if dom in alg:
+        roof["achieved"] = alg[dom] / cls_ms[dom] / 1e6
+        roof["frac"] = roof["achieved"] / peak
+        roof["algorithmic_bytes_per_step"] = alg[dom]
+    else:
+        roof["achieved"] = None
+        roof["frac"] = None
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+           "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": B,
+                      "prompt_lengths": [int(lens.min()), int(lens.max())], "mask": list(wl["mask"]),
+                      "skip_fraction": float(1 - mask.mean()), "l2": "inputs larger than L2 (weights + KV >> 126 MB)",
+                      "parallelism": "replicas" if world > 1 else "single"},
+           "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+           "roofline": roof,
+           "step_roofline": {"bytes_strict": bm["strict"], "bytes_full": bm["full"],
+                             "frac_strict_of_measured": bm["strict"] / (ms_step * 1e6) / peak,
+                             "frac_full_of_measured": bm["full"] / (ms_step * 1e6) / peak,
+                             "frac_strict_of_8TBps": bm["strict"] / (ms_step * 1e6) / 8000.0,
+                             "floor_ms_strict_measured_peak": bm["strict"] / peak / 1e6},
+           "dense": {"ms_per_step": dense_ms, "bytes_strict": bm_dense["strict"],
+                     "latency_ratio_routed_over_dense": ms_step / dense_ms,
+                     "bytes_ratio_routed_over_dense": bm["full"] / bm_dense["full"]},
+           "kernel_ms_per_step": cls_ms, "route": route}
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5)
+        out["cpu_baseline"].pop("ms_per_step", None)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg2_8b_b32", choices=sorted(WORKLOADS))
+    ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-route", action="store_true")
+    args = ap.parse_args()
+    wl = dict(WORKLOADS[args.workload])
+    if args.mask:
+        parts = args.mask.split(":")
+        wl["mask"] = tuple([parts[0]] + [float(x) for x in parts[1:]])
+    if args.steps is None:
+        args.steps = 64 if args.impl == "cuda" else 2
+    if args.impl == "reference" and args.warmup > 1:
+        args.warmup = 1
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    shape = SHAPES[wl["shape"]]
+    rank = int(os.environ.get("RANK", "0"))
+    lens = fi.prompt_lengths(wl["B"], wl["lo"], wl["hi"], 1000 + rank)
+    mask = make_mask(wl["mask"], wl["B"], shape.n_layers, 2000 + rank)
+    if args.impl == "reference":
+        run_reference(args, wl, shape, mask, lens)
+    else:
+        run_cuda(args, wl, shape, mask, lens)
+
+
+if __name__ == "__main__":
+    main()
