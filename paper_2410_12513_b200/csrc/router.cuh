@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) router_token_scores(const HT* __restrict_
 
 // Pass 2: one block per sequence; float64 mean in a fixed order (strided partial sums
 // then a fixed tree), sigmoid for mode 1, threshold with ">=".
-__global__ void __launch_bounds__(256) router_finalize(const float* __restrict__ tok, const int32_t* __restrict__ cu,
+static __global__ void __launch_bounds__(256) router_finalize(const float* __restrict__ tok, const int32_t* __restrict__ cu,
                                                        int L, int layer, int mode, float tau,
                                                        uint8_t* __restrict__ mask, float* __restrict__ scores,
                                                        uint32_t* __restrict__ flags) {
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(256) router_finalize(const float* __restrict__
 // gives the keep bits, popc of the lower lanes the position inside the chunk, a running
 // base the position in the list.  idx[l] = ascending active rows (rest -1), cnt[l],
 // slot[l][b] = position of b in idx[l] or -1.
-__global__ void __launch_bounds__(32) plan_compact(const uint8_t* __restrict__ mask, int B, int L,
+static __global__ void __launch_bounds__(32) plan_compact(const uint8_t* __restrict__ mask, int B, int L,
                                                    int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
                                                    int32_t* __restrict__ slot, uint32_t* __restrict__ flags) {
     const int l = blockIdx.x, lane = threadIdx.x;
