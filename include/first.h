@@ -143,6 +143,41 @@ int first_prefill_route(first_ctx *ctx, int32_t layer, const void *hidden, int32
                         const float *router_b, float tau, int32_t mode, uint8_t *mask, float *scores,
                         void *stream);
 
+/* The router call for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of first_prefill_route, same arithmetic, same
+ * kernels, same results.)
+ *
+ * Who needs it: first_prefill_route takes its per-token scratch from a context, and
+ * creating a context calls cudaMalloc.  Some hosts cannot do that at the point where they
+ * want to route a batch: a serving process whose framework allocator has already reserved
+ * the whole GPU, so that a raw cudaMalloc fails; a plugin that runs under a fixed memory
+ * budget it may not exceed; code on a latency-critical path where cudaMalloc's implicit
+ * device-wide synchronisation is not acceptable.  This entry point needs no context and
+ * calls no cudaMalloc, cudaFree or other allocating routine.  Its scratch is a fixed array
+ * compiled into the library image: FIRST_STATIC_ROUTE_MAX_TOKENS float32 token scores plus
+ * a 256-byte header (4 MiB + 256 B).  Every GPU on which a process loads this library
+ * holds that array until the process exits, whether or not this call is ever used.
+ *
+ * Arguments are those of first_prefill_route, with n_layers and d_model passed directly
+ * (d_model a multiple of 8, at most 12288) and
+ *   flags   dev uint32 [1] or NULL: receives FIRST_FLAG_EMPTY_SEQ (OR-ed in, never cleared
+ *           here).  With NULL a word inside the built-in scratch is used; it is reset to
+ *           zero at the start of every call and cannot be read back by the caller.
+ * Limits and rules:
+ *   - total_tokens > FIRST_STATIC_ROUTE_MAX_TOKENS returns FIRST_E_CAPACITY, nothing runs.
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.
+ *     Token scores are fully rewritten before they are read, so stale contents are harmless,
+ *     but two calls whose kernels overlap on the GPU (different streams, or different host
+ *     threads on different streams) race on it: keep calls on one stream, or order them.
+ * Errors: FIRST_E_ARG, FIRST_E_UNSUPPORTED (d_model), FIRST_E_CAPACITY, FIRST_E_CUDA. */
+#define FIRST_STATIC_ROUTE_MAX_TOKENS 1048576
+int first_prefill_route_static(int32_t layer, int32_t n_layers, int32_t d_model, const void *hidden,
+                               int32_t hidden_dtype, const int32_t *cu_seqlens, int32_t B, int64_t total_tokens,
+                               const float *router_w, const float *router_b, float tau, int32_t mode,
+                               uint8_t *mask, float *scores, uint32_t *flags, void *stream);
+
 /* Fix the skip mask of the current batch and build, per layer, the ascending list of
  * rows that keep it (one decision per sequence per layer, "Adaptive Router Module";
  * fixed for all decode steps, "Inference for FiRST" item 2).  Must be called before

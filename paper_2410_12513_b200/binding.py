@@ -60,6 +60,10 @@ def lib():
         L.first_prefill_route.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
                                           C.c_int64, C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
+        L.first_prefill_route_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                                 C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_float, C.c_int32,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.first_prefill_route_static.restype = C.c_int
         L.first_set_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.first_get_plan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(KVCacheC), C.c_void_p, C.c_void_p,
@@ -161,6 +165,23 @@ def first_prefill_route(h, layer, hidden, cu_seqlens, router_w, router_b, tau, m
                                    _stream(stream))
     if rc:
         raise FirstError(rc, "first_prefill_route")
+
+
+def first_prefill_route_static(layer, n_layers, hidden, cu_seqlens, router_w, router_b, tau, mode, mask,
+                               scores=None, flags=None, stream=None):
+    """Context-free router call that allocates nothing (built-in scratch of
+    FIRST_STATIC_ROUTE_MAX_TOKENS token scores); see first.h for the limits."""
+    if hidden.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("hidden must be float32 or bfloat16")
+    hd = FIRST_DTYPE_F32 if hidden.dtype == torch.float32 else FIRST_DTYPE_BF16
+    rc = lib().first_prefill_route_static(int(layer), int(n_layers), hidden.shape[1], _dev(hidden, None, "hidden"), hd,
+                                          _dev(cu_seqlens, torch.int32, "cu_seqlens"), cu_seqlens.numel() - 1,
+                                          hidden.shape[0], _dev(router_w, torch.float32, "router_w"),
+                                          _dev(router_b, torch.float32, "router_b"), float(tau), int(mode),
+                                          _dev(mask, torch.uint8, "mask"), _dev(scores, torch.float32, "scores"),
+                                          _dev(flags, torch.int32, "flags"), _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_prefill_route_static")
 
 
 def first_set_mask(h, mask, stream=None):
