@@ -5,9 +5,12 @@
 #include <new>
 #include <vector>
 
+#include <type_traits>
+
 #include "attn_simple.cuh"
 #include "common.cuh"
 #include "first.h"
+#include "gemm_tc.cuh"
 #include "gemv.cuh"
 #include "router.cuh"
 #include "step.cuh"
@@ -43,6 +46,11 @@ struct first_ctx {
     // scratch (device)
     float *x = nullptr, *xn = nullptr, *qkv = nullptr, *q = nullptr, *att = nullptr, *gu = nullptr, *act = nullptr;
     float *o_part = nullptr, *logits_int = nullptr, *tokscore = nullptr;
+    __nv_bfloat16 *xh = nullptr, *xl = nullptr, *acth = nullptr, *actl = nullptr;  // hi/lo activation splits
+    // TMA descriptors of the weight matrices (bf16 models)
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
+    CUtensorMap tm_lm{};
+    bool tc_ready = false;
     float2 *ml_part = nullptr, *cs = nullptr;
     double* inv_freq = nullptr;
     int32_t *idx = nullptr, *cnt = nullptr, *slot = nullptr;
@@ -63,6 +71,7 @@ struct first_ctx {
     // options
     int max_gemv_rows = -1;
     int attn_simple = -1;
+    int tc_use_lo = 1;
 };
 
 namespace {
@@ -104,6 +113,116 @@ struct Launch {
 
 int check_launch(first_ctx*) {
     CU_TRY(cudaGetLastError());
+    return FIRST_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// 2-D bfloat16 row-major matrix [rows][cols] -> TMA descriptor with a [box_rows][64] box in
+// 128-byte-swizzled rows; out-of-range elements read as zero.
+int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, bool weights) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return FIRST_E_CUDA;
+    if ((reinterpret_cast<uintptr_t>(ptr) & 15u) || (cols * 2) % 16) return FIRST_E_UNSUPPORTED;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)tc::kBlockK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    weights ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        std::snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "cuTensorMapEncodeTiled failed with %d", (int)r);
+        return FIRST_E_CUDA;
+    }
+    return FIRST_OK;
+}
+
+constexpr int kTcSmemMax = 227 * 1024;
+
+// Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
+//   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
+//   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
+int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_out, int K,
+                   const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
+                   const int32_t* idx) {
+    int rc;
+    for (int r0 = 0; r0 < m; r0 += 256) {
+        const int mm = std::min(256, m - r0);
+        tc::GemmParams p{};
+        p.n_out = n_out; p.K = K; p.m = mm;
+        p.n_pad = (mm + 15) / 16 * 16;
+        p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+        p.use_lo = c->tc_use_lo ? 1 : 0;
+        const int tiles = (n_out + tc::kBlockM - 1) / tc::kBlockM;
+        int ksplit = 1;
+        if (epi != tc::kEpiStore) {
+            ksplit = (2 * c->n_sm + tiles / 2) / tiles;
+            ksplit = std::max(1, std::min(ksplit, p.kblocks / 4));
+        }
+        p.ksplit = std::max(1, ksplit);
+        const int stage_bytes = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
+        const int budget = (3 * stage_bytes <= 110 * 1024) ? 110 * 1024 : 200 * 1024;
+        p.stages = std::max(1, std::min(8, budget / stage_bytes));
+        int cols = 32;
+        while (cols < p.n_pad) cols *= 2;
+        p.tmem_cols = cols;
+        p.Y = Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy);
+        p.ldy = ldy;
+        p.idx = idx ? idx + r0 : nullptr;
+        p.flags = c->flags;
+        CUtensorMap tmBh, tmBl;
+        if ((rc = make_map(&tmBh, Xh + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
+        if ((rc = make_map(&tmBl, Xl + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
+        const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 8 * (2 * p.stages + 1) + 64;
+        int e = epi;
+        if (e == tc::kEpiAtomic) {
+            if (p.ksplit == 1) e = tc::kEpiStore;
+            else CU_TRY(cudaMemsetAsync(p.Y, 0, (size_t)mm * ldy * sizeof(float), st));
+        }
+        const int grid = tiles * p.ksplit;
+        if (e == tc::kEpiStore)
+            FIRST_LAUNCH(kClsGemmTc, (tc::gemm_tc_kernel<tc::kEpiStore><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
+        else if (e == tc::kEpiAtomic)
+            FIRST_LAUNCH(kClsGemmTc, (tc::gemm_tc_kernel<tc::kEpiAtomic><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
+        else
+            FIRST_LAUNCH(kClsGemmTc,
+                         (tc::gemm_tc_kernel<tc::kEpiScatterAtomic><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
+        if ((rc = check_launch(c))) return rc;
+    }
+    return FIRST_OK;
+}
+
+int tc_setup(first_ctx* c) {
+    const first_model_desc& d = c->d;
+    int rc;
+    const int L = d.n_layers;
+    c->tm_wqkv.resize(L); c->tm_wo.resize(L); c->tm_wgu.resize(L); c->tm_wd.resize(L);
+    for (int l = 0; l < L; ++l) {
+        if ((rc = make_map(&c->tm_wqkv[l], c->wqkv[l], c->qkvd, d.d_model, tc::kBlockM, true)) ||
+            (rc = make_map(&c->tm_wo[l], c->wo[l], d.d_model, c->qd, tc::kBlockM, true)) ||
+            (rc = make_map(&c->tm_wgu[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, tc::kBlockM, true)) ||
+            (rc = make_map(&c->tm_wd[l], c->w_down[l], d.d_model, d.ffn_dim, tc::kBlockM, true)))
+            return rc;
+    }
+    if ((rc = make_map(&c->tm_lm, c->lm_head, d.vocab, d.d_model, tc::kBlockM, true))) return rc;
+    CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiScatterAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
+    c->tc_ready = true;
     return FIRST_OK;
 }
 
@@ -157,15 +276,35 @@ int launch_attn_simple(first_ctx* c, cudaStream_t st, int S, int m, const void* 
     }
 }
 
+// One projection of m compact rows: tensor cores when the row count makes it a dense
+// contraction (bf16 weights), the CUDA-core GEMV otherwise.
+//   out_mode 0: Y[j][f] = ..   (compact rows, row stride ldy)
+//   out_mode 1: Y[idx[j]][f] += ..   (scatter-add into the residual stream)
+template <typename WT>
+int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUtensorMap* tm, int n_out, int K,
+            const float* X, const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int out_mode, float* Y,
+            int64_t ldy, const int32_t* idx, bool allow_split = true) {
+    if (use_tc) {
+        const int epi = out_mode == 1 ? tc::kEpiScatterAtomic : (allow_split ? tc::kEpiAtomic : tc::kEpiStore);
+        return launch_gemm_tc(c, st, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx);
+    }
+    if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx);
+    return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
+}
+
 // The whole step, for one weight/cache element type.
 template <typename WT>
 int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* kv, float* logits,
                      int32_t* next_tokens, float* layer_inputs, cudaStream_t st) {
     const first_model_desc& d = c->d;
     const int B = c->B, D = d.d_model, F = d.ffn_dim, V = d.vocab, L = d.n_layers, hd = d.head_dim;
+    constexpr bool kBf16 = std::is_same<WT, __nv_bfloat16>::value;
+    const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 2;
+    auto tc_for = [&](int m) { return kBf16 && c->tc_ready && m > gemv_max; };
     int rc;
-    FIRST_LAUNCH(kClsStepBegin, (step_begin<WT><<<B, 256, 0, st>>>(tokens, static_cast<const WT*>(c->embed), D, V, kv->pos, c->inv_freq, hd / 2,
-                                      c->x, c->cs, c->flags)));
+    FIRST_LAUNCH(kClsStepBegin, (step_begin<WT><<<B, 256, 0, st>>>(tokens, static_cast<const WT*>(c->embed), D, V,
+                                                                   kv->pos, c->inv_freq, hd / 2, c->x, c->cs,
+                                                                   c->flags)));
     if ((rc = check_launch(c))) return rc;
 
     int S = (d.max_tokens_per_seq + 255) / 256;
@@ -178,27 +317,44 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                                    cudaMemcpyDeviceToDevice, st));
         const int m = c->cnt_h[l];
         if (m == 0) continue;  // every sequence skips this layer: no launch at all
+        const bool t = tc_for(m);
         const int32_t* idx = c->idx + (size_t)l * B;
         int32_t* len_l = kv->len + (size_t)l * B;
+        float* f32 = t ? nullptr : c->xn;
+        __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
         // attention half
-        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->attn_norm[l], d.rms_eps, c->xn, nullptr, nullptr)));
+        FIRST_LAUNCH(kClsRmsnorm,
+                     (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->attn_norm[l], d.rms_eps, f32, xh, xl)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_gemv<WT, kStore>(c, st, c->wqkv[l], c->qkvd, D, c->xn, m, c->qkv, c->qkvd, nullptr))) return rc;
-        FIRST_LAUNCH(kClsRopeAppend, (rope_append<WT><<<m, 256, 0, st>>>(c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
-                                           static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total,
-                                           kv->slab_off, kv->slab_cap, len_l, c->flags)));
+        if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
+                              c->qkv, c->qkvd, nullptr)))
+            return rc;
+        FIRST_LAUNCH(kClsRopeAppend,
+                     (rope_append<WT><<<m, 256, 0, st>>>(c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
+                                                         static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]),
+                                                         kv->cap_total, kv->slab_off, kv->slab_cap, len_l, c->flags)));
         if ((rc = check_launch(c))) return rc;
         if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
-        FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd, c->att, nullptr, nullptr)));
+        FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd,
+                                                                                     t ? nullptr : c->att, xh, xl)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_gemv<WT, kScatterAdd>(c, st, c->wo[l], D, c->qd, c->att, m, c->x, D, idx))) return rc;
+        if ((rc = project<WT>(c, st, t, c->wo[l], t ? &c->tm_wo[l] : nullptr, D, c->qd, c->att, c->xh, c->xl, m, 1, c->x,
+                              D, idx)))
+            return rc;
         // feed-forward half
-        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->ffn_norm[l], d.rms_eps, c->xn, nullptr, nullptr)));
+        FIRST_LAUNCH(kClsRmsnorm,
+                     (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->ffn_norm[l], d.rms_eps, f32, xh, xl)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_gemv<WT, kStore>(c, st, c->w_gate_up[l], 2 * F, D, c->xn, m, c->gu, 2 * F, nullptr))) return rc;
-        FIRST_LAUNCH(kClsSiluMul, (silu_mul<<<std::min((m * F + 255) / 256, c->n_sm * 8), 256, 0, st>>>(c->gu, m, F, c->act, nullptr, nullptr)));
+        if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl, m,
+                              0, c->gu, 2 * F, nullptr)))
+            return rc;
+        FIRST_LAUNCH(kClsSiluMul, (silu_mul<<<std::min((m * F + 255) / 256, c->n_sm * 8), 256, 0, st>>>(
+                                      c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr,
+                                      t ? c->actl : nullptr)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_gemv<WT, kScatterAdd>(c, st, c->w_down[l], D, F, c->act, m, c->x, D, idx))) return rc;
+        if ((rc = project<WT>(c, st, t, c->w_down[l], t ? &c->tm_wd[l] : nullptr, D, F, c->act, c->acth, c->actl, m, 1,
+                              c->x, D, idx)))
+            return rc;
     }
     float* lg = logits;
     if (!lg && next_tokens) {
@@ -206,9 +362,14 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         lg = c->logits_int;
     }
     if (lg) {
-        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<B, 256, 0, st>>>(c->x, nullptr, D, c->final_norm, d.rms_eps, c->xn, nullptr, nullptr)));
+        const bool t = tc_for(B);
+        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<B, 256, 0, st>>>(c->x, nullptr, D, c->final_norm, d.rms_eps,
+                                                                   t ? nullptr : c->xn, t ? c->xh : nullptr,
+                                                                   t ? c->xl : nullptr)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_gemv<WT, kStore>(c, st, c->lm_head, V, D, c->xn, B, lg, V, nullptr))) return rc;
+        if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
+                              nullptr, false)))
+            return rc;
     }
     FIRST_LAUNCH(kClsStepEnd, (step_end<<<B, 256, 0, st>>>(lg, V, next_tokens, kv->pos)));
     return check_launch(c);
@@ -287,6 +448,12 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         (rc = dev_alloc(&c->idx, MB * d.n_layers)) || (rc = dev_alloc(&c->cnt, (size_t)d.n_layers)) ||
         (rc = dev_alloc(&c->slot, MB * d.n_layers)) || (rc = dev_alloc(&c->flags, (size_t)1)))
         return fail(rc);
+    if (d.dtype == FIRST_DTYPE_BF16) {
+        if ((rc = dev_alloc(&c->xh, MB * xw)) || (rc = dev_alloc(&c->xl, MB * xw)) ||
+            (rc = dev_alloc(&c->acth, MB * d.ffn_dim)) || (rc = dev_alloc(&c->actl, MB * d.ffn_dim)))
+            return fail(rc);
+        if ((rc = tc_setup(c))) return fail(rc);
+    }
     c->tok_cap = (int64_t)d.max_batch * d.max_tokens_per_seq;
     if ((rc = dev_alloc(&c->tokscore, (size_t)c->tok_cap))) return fail(rc);
     std::vector<double> inv(d.head_dim / 2);
@@ -301,7 +468,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
 int first_destroy(first_ctx* c) {
     if (!c) return FIRST_OK;
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
-                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags};
+                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -422,6 +589,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     if (!c || !name) return FIRST_E_ARG;
     if (!std::strcmp(name, "max_gemv_rows")) c->max_gemv_rows = (int)value;
     else if (!std::strcmp(name, "attn_simple")) c->attn_simple = (int)value;
+    else if (!std::strcmp(name, "tc_use_lo")) c->tc_use_lo = value != 0;
     else return FIRST_E_ARG;
     return FIRST_OK;
 }

@@ -1,0 +1,238 @@
+// Tensor-core projection path (tcgen05 + TMEM + TMA) for layers with enough active rows
+// to make the projection a dense contraction:  Y[j][f] (+)= sum_k W[f][k] * X[j][k].
+//
+// "Swap-AB": the weight matrix is the 128-row M operand, streamed once from HBM by TMA into
+// 128-byte-swizzled shared memory; the compacted activations (m rows, padded to a multiple
+// of 16) are the N operand; the float32 accumulator tile [128 features][N rows] lives in
+// tensor memory.  Activations arrive as a bfloat16 hi/lo pair (x = hi + lo to 2^-17), and
+// each weight tile is multiplied by both halves into the same accumulator, so the result
+// keeps float32-grade activations while the weights stay bfloat16.
+//
+// Work unit = (128-feature tile, K range).  With several K ranges per tile the partial sums
+// meet in global memory through float32 reductions (red.global.add).
+// Roles inside a CTA of 6 warps: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = epilogue (one TMEM lane quadrant each).  Every wait is bounded.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "first.h"
+
+namespace first {
+namespace tc {
+
+constexpr int kBlockM = 128;  // weight rows (output features) per tile
+constexpr int kBlockK = 64;   // bf16 elements per 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kABytes = kBlockM * kBlockK * 2;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+enum Epilogue { kEpiStore = 0, kEpiAtomic = 1, kEpiScatterAtomic = 2 };
+
+struct GemmParams {
+    int n_out, K, m, n_pad;
+    int kblocks, ksplit;
+    int stages, tmem_cols, use_lo;
+    float* Y;
+    int64_t ldy;
+    const int32_t* idx;
+    uint32_t* flags;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or when another role already gave up),
+// raising the CTA's abort word and the device flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_s, uint32_t* flags) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_s) return false;
+    }
+    *abort_s = 1;
+    atomicOr(flags, FIRST_FLAG_WAIT_EXPIRED);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major operand in 128-byte-swizzled rows:
+// start address >> 4, stride between 8-row groups = 1024 bytes, descriptor version 1,
+// swizzle mode 2 (128 B).  The leading-dimension field is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: D = f32, A = B = bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Dynamic shared memory: [stages][A 16 KB | B_hi n_pad*128 | B_lo n_pad*128] (1024-aligned), then barriers.
+template <int EPI>
+__global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                      const __grid_constant__ CUtensorMap tmBh,
+                                                      const __grid_constant__ CUtensorMap tmBl, const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int b_bytes = p.n_pad * 128;
+    const int stage_bytes = kABytes + b_bytes * (p.use_lo ? 2 : 1);
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;  // full[S], empty[S], tmem_full : 8 B each
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (p.stages + s); };
+    const uint32_t tmem_full_bar = bars + 16u * p.stages;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x / p.ksplit, split = blockIdx.x - tile * p.ksplit;
+    const int kb0 = (int)((int64_t)p.kblocks * split / p.ksplit), kb1 = (int)((int64_t)p.kblocks * (split + 1) / p.ksplit);
+    const int nkb = kb1 - kb0;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBh) : "memory");
+        if (p.use_lo) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBl) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_base_s;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            const uint32_t tx = (uint32_t)stage_bytes;
+            int issued = 0;
+            for (int i = 0; i < nkb; ++i, ++issued) {
+                const int s = i % p.stages;
+                const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, &abort_s, p.flags)) break;
+                const uint32_t sa = base + (uint32_t)s * stage_bytes;
+                mbar_expect_tx(full_bar(s), tx);
+                const int kc = (kb0 + i) * kBlockK;
+                tma_load_2d_hint(sa, &tmA, full_bar(s), kc, tile * kBlockM, pol_stream);
+                tma_load_2d(sa + kABytes, &tmBh, full_bar(s), kc, 0);
+                if (p.use_lo) tma_load_2d(sa + kABytes + b_bytes, &tmBl, full_bar(s), kc, 0);
+            }
+            if (abort_s) {
+                // let the copies already issued land before this CTA's shared memory goes away
+                for (int i = max(0, issued - p.stages); i < issued; ++i) {
+                    const uint32_t bar = full_bar(i % p.stages), ph = (uint32_t)(i / p.stages) & 1u;
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, ph); ++it) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(p.n_pad);
+            bool ok = true;
+            for (int i = 0; i < nkb && ok; ++i) {
+                const int s = i % p.stages;
+                const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+                ok = mbar_wait(full_bar(s), ph, &abort_s, p.flags);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = base + (uint32_t)s * stage_bytes;
+                const uint64_t da = smem_desc_sw128(sa), dbh = smem_desc_sw128(sa + kABytes);
+#pragma unroll
+                for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                    umma_bf16(tmem_d, da + 2u * k, dbh + 2u * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (p.use_lo) {
+                    const uint64_t dbl = smem_desc_sw128(sa + kABytes + b_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) umma_bf16(tmem_d, da + 2u * k, dbl + 2u * k, idesc, 1u);
+                }
+                umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+            }
+            umma_commit(tmem_full_bar);  // accumulator complete (arrives even after a failed wait)
+        }
+    } else {
+        const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok && nkb > 0) {
+            const int quad = warp & 3;
+            const int f = tile * kBlockM + quad * 32 + lane;
+            const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
+            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(lane_addr + (uint32_t)c0, v);
+                if (f < p.n_out) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const int j = c0 + c;
+                        if (j < p.m) {
+                            const float val = __uint_as_float(v[c]);
+                            if (EPI == kEpiStore) p.Y[(size_t)j * p.ldy + f] = val;
+                            else if (EPI == kEpiAtomic) atomicAdd(p.Y + (size_t)j * p.ldy + f, val);
+                            else atomicAdd(p.Y + (size_t)p.idx[j] * p.ldy + f, val);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+    }
+}
+
+}  // namespace tc
+}  // namespace first
