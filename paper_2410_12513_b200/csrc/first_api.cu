@@ -151,7 +151,7 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
     return FIRST_OK;
 }
 
-constexpr int kTcSmemMax = 227 * 1024;
+constexpr int kTcSmemMax = 210 * 1024;
 
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
 //   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
