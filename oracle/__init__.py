@@ -53,7 +53,7 @@ def build(force: bool = False) -> Path:
 class _Model(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "ffn_dim", "vocab",
-                 "weight_dtype")] + [("rope_base", C.c_double), ("rms_eps", C.c_double)]
+                 "weight_dtype")] + [("rope_base", C.c_double), ("rms_eps", C.c_double), ("kv_dtype", C.c_int32)]
 
 
 class _Weights(C.Structure):
@@ -119,7 +119,8 @@ class OracleModel:
     are float32.
     """
 
-    def __init__(self, shape: Shape, weights: dict):
+    def __init__(self, shape: Shape, weights: dict, kv_bf16=None):
+        """kv_bf16: cache storage format; default = bfloat16 iff the weights are bfloat16."""
         self.shape = shape
         L = shape.n_layers
         keep = {}
@@ -150,8 +151,9 @@ class OracleModel:
         self._keep = keep
         self._arrs = {k: _ptr_array(keep[k]) for k in
                       ("attn_norm", "ffn_norm", "wq", "wk", "wv", "wo", "wg", "wu", "wd")}
+        self.kv_dtype = self.weight_dtype if kv_bf16 is None else int(bool(kv_bf16))
         self.c_model = _Model(s.n_layers, s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn_dim,
-                              s.vocab, self.weight_dtype, float(s.rope_base), float(s.rms_eps))
+                              s.vocab, self.weight_dtype, float(s.rope_base), float(s.rms_eps), self.kv_dtype)
         self.c_weights = _Weights(keep["embed"].ctypes.data, keep["lm_head"].ctypes.data,
                                   keep["final_norm"].ctypes.data,
                                   *[C.cast(self._arrs[k], C.POINTER(C.c_void_p)) for k in

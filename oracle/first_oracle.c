@@ -14,6 +14,10 @@
  * so the oracle's own rounding is far below the tolerances it is used to judge.
  * Weight matrices may be handed in as float32 or as bfloat16 bit patterns (uint16,
  * the upper half of the float32 word); bfloat16 values are widened exactly.
+ * The KV cache has a storage format too (kv_dtype): float32, or bfloat16, in which case a
+ * key/value is rounded to bfloat16 once, when it enters the cache, and attention reads the
+ * rounded value -- the same contract as for weights: both sides agree on the stored values,
+ * all arithmetic on them stays float32/float64.
  *
  * What follows the paper, and where:
  *   - layer recursion  H_i = H_{i-1} + phi_i(H^1..H^j)             Eq. 1 (Problem Statement)
@@ -49,6 +53,8 @@ typedef struct {
     int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, ffn_dim, vocab;
     int32_t weight_dtype; /* 0 = float32, 1 = bfloat16 bit patterns (uint16) */
     double rope_base, rms_eps;
+    int32_t kv_dtype;     /* storage format of cached keys/values: 0 = float32, 1 = values rounded to
+                             bfloat16 (nearest even) when stored, still held in float32 words */
 } fo_model;
 
 typedef struct {
@@ -76,6 +82,22 @@ typedef struct {
     int32_t *len;            /* [L][B] tokens present */
     int32_t *pos;            /* [B] absolute index of the next token */
 } fo_kv;
+
+/* float32 -> nearest bfloat16 (ties to even), returned widened back to float32 */
+static inline float bf16_round(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7f800000u) == 0x7f800000u) return f; /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+static void store_round(float *v, size_t n, int kv_dtype) {
+    if (kv_dtype == 1)
+        for (size_t i = 0; i < n; ++i) v[i] = bf16_round(v[i]);
+}
 
 static inline float bf16_widen(uint16_t h) {
     uint32_t u = ((uint32_t)h) << 16;
@@ -258,6 +280,8 @@ int fo_decode_step(const fo_model *m, const fo_weights *w, int32_t B, const int3
             linear(w->wv[l], dt, (int)kvd, D, xn, (size_t)D, Vc + (size_t)T * kvd, kvd, 1);
             rope(q, Hq, hd, kv->pos[b], m->rope_base);
             rope(Kc + (size_t)T * kvd, Hkv, hd, kv->pos[b], m->rope_base);
+            store_round(Kc + (size_t)T * kvd, kvd, m->kv_dtype); /* the cache's storage format */
+            store_round(Vc + (size_t)T * kvd, kvd, m->kv_dtype);
             kv->len[(size_t)l * B + b] = T + 1;
             attend(m, q, Kc, Vc, T + 1, att, score);
             linear(w->wo[l], dt, D, (int)qd, att, qd, proj, (size_t)D, 1);
@@ -326,6 +350,8 @@ int fo_forward_full(const fo_model *m, const fo_weights *w, int32_t n_total, con
             rope(Q + (size_t)j * qd, Hq, hd, j, m->rope_base);
             rope(K + (size_t)j * kvd, Hkv, hd, j, m->rope_base);
         }
+        store_round(K, (size_t)r * kvd, m->kv_dtype); /* attention reads what the cache would hold */
+        store_round(Vv, (size_t)r * kvd, m->kv_dtype);
         if (k_out && k_out[l]) memcpy(k_out[l], K, (size_t)r * kvd * sizeof(float));
         if (v_out && v_out[l]) memcpy(v_out[l], Vv, (size_t)r * kvd * sizeof(float));
 #pragma omp parallel

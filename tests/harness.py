@@ -9,8 +9,8 @@ import oracle
 
 
 # ------------------------------------------------------------------ oracle side
-def oracle_model(shape, weights):
-    return oracle.OracleModel(oracle.Shape(**shape.asdict()), weights)
+def oracle_model(shape, weights, kv_bf16=None):
+    return oracle.OracleModel(oracle.Shape(**shape.asdict()), weights, kv_bf16)
 
 
 def widen(a):

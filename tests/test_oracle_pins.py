@@ -280,8 +280,40 @@ def test_bf16_weights_are_widened_exactly():
     wb = fi.make_weights(s, 8, True)
     wf = {k: ([fi.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a for a in v] if isinstance(v, list)
               else (fi.bf16_bits_to_f32(v) if v.dtype == np.uint16 else v)) for k, v in wb.items()}
-    mb = oracle.OracleModel(oracle.Shape(**s.asdict()), wb)
-    mf = oracle.OracleModel(oracle.Shape(**s.asdict()), wf)
+    mb = oracle.OracleModel(oracle.Shape(**s.asdict()), wb, kv_bf16=False)
+    mf = oracle.OracleModel(oracle.Shape(**s.asdict()), wf, kv_bf16=False)
     assert mb.weight_dtype == 1 and mf.weight_dtype == 0
     toks = fi.tokens(s, 6, 2)
     assert np.array_equal(oracle.forward_full(mb, toks)["logits"], oracle.forward_full(mf, toks)["logits"])
+
+
+def test_bf16_cache_storage_rounds_once_like_torch():
+    """kv_dtype = bfloat16: keys/values are rounded to bfloat16 when they enter the cache (nearest,
+    ties to even -- checked against torch's conversion) and attention reads the rounded values;
+    nothing else changes.  Layer 0 sees identical inputs in both modes, so its stored keys are the
+    rounded float32-mode keys exactly."""
+    torch = pytest.importorskip("torch")
+    s = fi.TINY_GQA
+    wb = fi.make_weights(s, 8, True)
+    m32 = oracle.OracleModel(oracle.Shape(**s.asdict()), wb, kv_bf16=False)
+    m16 = oracle.OracleModel(oracle.Shape(**s.asdict()), wb)  # default: cache format follows the weights
+    assert m32.kv_dtype == 0 and m16.kv_dtype == 1
+    toks = fi.tokens(s, 12, 3)
+    a = oracle.forward_full(m32, toks, want_kv=True, logits_from=0)
+    b = oracle.forward_full(m16, toks, want_kv=True, logits_from=0)
+    rnd = lambda x: torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(b["k"][0], rnd(a["k"][0])) and np.array_equal(b["v"][0], rnd(a["v"][0]))
+    for l in range(s.n_layers):
+        assert np.array_equal(b["k"][l], rnd(b["k"][l])) and np.array_equal(b["v"][l], rnd(b["v"][l]))
+    d = np.abs(a["logits"] - b["logits"]).max() / (a["logits"].max() - a["logits"].min())
+    assert 0 < d < 2e-2
+    # cached decode in bf16-cache mode still equals the cache-free recompute in the same mode
+    kv = oracle.OracleKV(m16.shape, [12])
+    oracle.prefill(m16, kv, 0, toks[:8])
+    keep = np.array([[1, 0, 1]], np.uint8)
+    cached = np.stack([oracle.decode_step(m16, toks[8 + t:9 + t], keep, kv)[0] for t in range(4)])
+    full = oracle.forward_full(m16, toks, n_prompt=8, keep=keep[0], logits_from=8)["logits"]
+    assert np.abs(cached - full).max() <= 1e-5
+    # ties round to even: 1 + 2^-8 is exactly between two bfloat16 values
+    tie = np.array([[1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8]], np.float32)
+    assert rnd(tie).tolist() == [[1.0, 1.015625]]
