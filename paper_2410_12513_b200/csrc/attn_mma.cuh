@@ -1,0 +1,288 @@
+// Grouped-query decode attention over the active rows' bfloat16 caches (head_dim 64/128).
+//
+// HBM-bound: every cached key and value of an active (sequence, kv head) is read once.
+// K/V tiles of 64 tokens are staged by TMA into 128-byte-swizzled shared memory through a
+// 3-stage ring (one producer warp, four consumer warps).  With 4..8 query heads per KV
+// head the score and PV products are too much arithmetic for the FP32 pipes at HBM speed
+// (about 4 FLOP per cache byte), so they run on the tensor cores via mma.sync m16n8k16:
+// the group's query heads are the M rows.  Precision: q and the softmax weights are split
+// into bfloat16 hi + lo; hi sits in rows 0..7 and lo in rows 8..15 of the same A fragment,
+// so one MMA yields both partial products and the thread adds them -- float32-grade q and p
+// against the stored bfloat16 keys/values.  Softmax is online, row maxima by quad shuffles.
+// The token axis is split in chunks of C tokens per CTA; attn_combine_var merges them.
+#pragma once
+#include "common.cuh"
+#include "first.h"
+#include "gemm_tc.cuh"  // mbarrier / TMA helpers
+
+namespace first {
+namespace attn {
+
+constexpr int kTile = 64;    // tokens per stage
+constexpr int kStages = 3;
+constexpr int kConsumers = 128;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// (x, y) -> packed bf16 hi parts and packed bf16 remainders
+__device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x - __low2float(h), y - __high2float(h));
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// grid (S_max, Hkv, m), 160 threads.  Work item = (active row i, kv head h, chunk c):
+// tokens [c*C, min(T, (c+1)*C)), T = len[b] (new token already appended).  Chunks past T exit.
+// q: [m][Hq][HD] float32, pre-scaled by 1/sqrt(HD).  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64x64.
+// o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum).
+template <int HD, int G>
+__global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
+                                                      const __grid_constant__ CUtensorMap tmV,
+                                                      const float* __restrict__ q, int64_t cap_total,
+                                                      const int64_t* __restrict__ slab_off,
+                                                      const int32_t* __restrict__ len_l,
+                                                      const int32_t* __restrict__ idx, int Hq, int C,
+                                                      float* __restrict__ o_part, float2* __restrict__ ml_part,
+                                                      uint32_t* __restrict__ flags) {
+    constexpr int kHalves = HD / 64;              // 128-byte column groups per row
+    constexpr int kBox = kTile * 128;             // bytes of one 64-token x 64-element box
+    constexpr int kStageBytes = 2 * kHalves * kBox;
+    constexpr int kKSteps = HD / 16, kNTiles = HD / 8;
+    static_assert(G <= 8, "query heads of a group are the 8 hi rows of the A fragment");
+
+    const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
+    const int b = idx[i];
+    const int T = len_l[b];
+    const int t_begin = c * C;
+    if (t_begin >= T) return;
+    const int t_end = min(T, t_begin + C);
+    const int n_tiles = (t_end - t_begin + kTile - 1) / kTile;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - tc::smem_u32(smem_raw));
+    __shared__ uint64_t bar_mem[2 * kStages];
+    __shared__ int abort_s;
+    auto full_bar = [&](int s) { return tc::smem_u32(&bar_mem[s]); };
+    auto empty_bar = [&](int s) { return tc::smem_u32(&bar_mem[kStages + s]); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == 4) {  // ---------------- producer
+        if (lane == 0) {
+            const int64_t row0 = (int64_t)h * cap_total + slab_off[b] + t_begin;
+            int issued = 0;
+            for (int j = 0; j < n_tiles; ++j, ++issued) {
+                const int s = j % kStages;
+                const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+                if (!tc::mbar_wait(empty_bar(s), ph ^ 1u, &abort_s, flags)) break;
+                const uint32_t sa = base + (uint32_t)s * kStageBytes;
+                tc::mbar_expect_tx(full_bar(s), kStageBytes);
+                const int row = (int)(row0 + (int64_t)j * kTile);
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                    tc::tma_load_2d(sa + hf * kBox, &tmK, full_bar(s), hf * 64, row);
+                    tc::tma_load_2d(sa + (kHalves + hf) * kBox, &tmV, full_bar(s), hf * 64, row);
+                }
+            }
+            if (abort_s) {
+                for (int j = max(0, issued - kStages); j < issued; ++j) {
+                    const uint32_t bar = full_bar(j % kStages), ph = (uint32_t)(j / kStages) & 1u;
+                    for (uint32_t it = 0; it < tc::kSpinLimit && !tc::mbar_try_wait(bar, ph); ++it) {}
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers: warp w owns tokens [16w, 16w+16) of every tile
+    const int g = lane >> 2, tq = lane & 3;
+    uint32_t qh[kKSteps][2], ql[kKSteps][2];  // A fragments: (k0..k0+1), (k0+8..k0+9) of row g
+    {
+        const float* qrow = q + ((size_t)i * Hq + (size_t)h * G + (g < G ? g : 0)) * HD;
+#pragma unroll
+        for (int ks = 0; ks < kKSteps; ++ks) {
+            float2 v0 = make_float2(0.f, 0.f), v1 = v0;
+            if (g < G) {
+                v0 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 2 * tq);
+                v1 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 8 + 2 * tq);
+            }
+            split2(v0.x, v0.y, qh[ks][0], ql[ks][0]);
+            split2(v1.x, v1.y, qh[ks][1], ql[ks][1]);
+        }
+    }
+    float o[kNTiles][4];
+#pragma unroll
+    for (int nt = 0; nt < kNTiles; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+    const int mat = lane >> 3, r8 = lane & 7;
+    bool ok = true;
+
+    for (int j = 0; j < n_tiles; ++j) {
+        const int s = j % kStages;
+        const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+        if (!tc::mbar_wait(full_bar(s), ph, &abort_s, flags)) { ok = false; break; }
+        const uint32_t sK = base + (uint32_t)s * kStageBytes, sV = sK + kHalves * kBox;
+        const int tile_t0 = t_begin + j * kTile;
+        const int valid = t_end - tile_t0;  // tokens of this tile that exist (may exceed 64)
+        if (valid < kTile) {
+            // rows past the end hold someone else's bytes: zero them in V so 0 * garbage stays 0
+            uint8_t* vptr = base_ptr + (size_t)s * kStageBytes + kHalves * kBox;
+            for (int e = lane; e < 16 * kHalves * 8; e += 32) {
+                const int row = warp * 16 + e / (kHalves * 8), cc = e % (kHalves * 8);
+                if (row >= valid)
+                    *reinterpret_cast<uint4*>(vptr + (cc >> 3) * kBox + row * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
+            }
+            __syncwarp();
+        }
+        // ---- scores S[g][token] for this warp's 16 tokens (two n-tiles of 8)
+        float sc[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < kKSteps; ++ks) {
+            const int row = warp * 16 + (mat >> 1) * 8 + r8;
+            const int cg = 2 * ks + (mat & 1);
+            const uint32_t addr = sK + (cg >> 3) * kBox + row * 128 + (((cg & 7) ^ (row & 7)) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(addr, b0, b1, b2, b3);
+            mma16816(sc[0], qh[ks][0], ql[ks][0], qh[ks][1], ql[ks][1], b0, b1);
+            mma16816(sc[1], qh[ks][0], ql[ks][0], qh[ks][1], ql[ks][1], b2, b3);
+        }
+        float sv[4];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int tok = warp * 16 + nt * 8 + 2 * tq + e;
+                const float v = (tok < valid) ? sc[nt][e] + sc[nt][e + 2] : -INFINITY;  // hi + lo parts
+                sv[nt * 2 + e] = v;
+                mx = fmaxf(mx, v);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        float p[4];
+        float scale = 1.f;
+        if (m_new == -INFINITY) {
+            p[0] = p[1] = p[2] = p[3] = 0.f;
+        } else {
+            scale = (m_run == -INFINITY) ? 0.f : __expf(m_run - m_new);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) p[e] = (sv[e] == -INFINITY) ? 0.f : __expf(sv[e] - m_new);
+        }
+        m_run = m_new;
+        l_run = l_run * scale + (p[0] + p[1] + p[2] + p[3]);
+#pragma unroll
+        for (int nt = 0; nt < kNTiles; ++nt) { o[nt][0] *= scale; o[nt][1] *= scale; o[nt][2] *= scale; o[nt][3] *= scale; }
+        uint32_t ph0, pl0, ph1, pl1;
+        split2(p[0], p[1], ph0, pl0);
+        split2(p[2], p[3], ph1, pl1);
+        // ---- O[g][d] += P[g][token] V[token][d]
+#pragma unroll
+        for (int n2 = 0; n2 < kNTiles / 2; ++n2) {
+            const int row = warp * 16 + (mat & 1) * 8 + r8;
+            const int cg = 2 * n2 + (mat >> 1);
+            const uint32_t addr = sV + (cg >> 3) * kBox + row * 128 + (((cg & 7) ^ (row & 7)) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4_t(addr, b0, b1, b2, b3);
+            mma16816(o[2 * n2], ph0, pl0, ph1, pl1, b0, b1);
+            mma16816(o[2 * n2 + 1], ph0, pl0, ph1, pl1, b2, b3);
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+    }
+
+    // ---- merge the four warps' partial softmax states through shared memory (stage memory is free now)
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    bar_consumers();
+    float* o_s = reinterpret_cast<float*>(base_ptr);       // [4][G][HD]
+    float* m_s = o_s + 4 * G * HD;                          // [4][G]
+    float* l_s = m_s + 4 * G;                               // [4][G]
+    if (g < G) {
+#pragma unroll
+        for (int nt = 0; nt < kNTiles; ++nt) {
+            float2 v = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
+            *reinterpret_cast<float2*>(o_s + ((size_t)warp * G + g) * HD + nt * 8 + 2 * tq) = v;
+        }
+        if (tq == 0) { m_s[warp * G + g] = m_run; l_s[warp * G + g] = l_run; }
+    }
+    bar_consumers();
+    if (!ok || abort_s) return;
+    for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
+        const int gg = e / HD, d = e - gg * HD;
+        const float M = fmaxf(fmaxf(m_s[gg], m_s[G + gg]), fmaxf(m_s[2 * G + gg], m_s[3 * G + gg]));
+        float acc = 0.f, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float mw = m_s[w * G + gg];
+            if (mw > -INFINITY) {
+                const float f = __expf(mw - M);
+                acc += o_s[((size_t)w * G + gg) * HD + d] * f;
+                l += l_s[w * G + gg] * f;
+            }
+        }
+        const size_t hq = (size_t)i * Hq + (size_t)h * G + gg;
+        o_part[(hq * S_max + c) * HD + d] = acc;
+        if (d == 0) ml_part[hq * S_max + c] = make_float2(M, l);
+    }
+}
+
+// Merge the chunks of each (row, query head); the number of chunks follows from the row's length.
+// out (float32) and/or its bfloat16 hi/lo split, [m][Hq*HD].
+__global__ void __launch_bounds__(128) attn_combine_var(const float* __restrict__ o_part,
+                                                        const float2* __restrict__ ml_part, int S_max, int HD, int Hq,
+                                                        int C, const int32_t* __restrict__ len_l,
+                                                        const int32_t* __restrict__ idx, float* __restrict__ out,
+                                                        __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    const size_t hq = blockIdx.x;
+    const int i = (int)(hq / Hq);
+    const int T = len_l[idx[i]];
+    const int S = min(S_max, (T + C - 1) / C);
+    float M = -INFINITY;
+    for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[hq * S_max + s].x);
+    float den = 0.f;
+    for (int s = 0; s < S; ++s) {
+        const float2 ml = ml_part[hq * S_max + s];
+        if (ml.x > -INFINITY) den += ml.y * __expf(ml.x - M);
+    }
+    for (int d = threadIdx.x; d < HD; d += blockDim.x) {
+        float o = 0.f;
+        for (int s = 0; s < S; ++s) {
+            const float mx = ml_part[hq * S_max + s].x;
+            if (mx > -INFINITY) o += o_part[(hq * S_max + s) * HD + d] * __expf(mx - M);
+        }
+        const float y = o / den;
+        if (out) out[hq * HD + d] = y;
+        if (hi) {
+            const __nv_bfloat16 hh = __float2bfloat16_rn(y);
+            hi[hq * HD + d] = hh;
+            lo[hq * HD + d] = __float2bfloat16_rn(y - __bfloat162float(hh));
+        }
+    }
+}
+
+}  // namespace attn
+}  // namespace first

@@ -6,7 +6,9 @@
 #include <vector>
 
 #include <type_traits>
+#include <unordered_map>
 
+#include "attn_mma.cuh"
 #include "attn_simple.cuh"
 #include "common.cuh"
 #include "first.h"
@@ -51,12 +53,15 @@ struct first_ctx {
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
     CUtensorMap tm_lm{};
     bool tc_ready = false;
+    struct KvMap { int64_t cap_total; CUtensorMap map; };
+    std::unordered_map<const void*, KvMap> kv_maps;  // TMA descriptors of cache tensors, by base pointer
     float2 *ml_part = nullptr, *cs = nullptr;
     double* inv_freq = nullptr;
     int32_t *idx = nullptr, *cnt = nullptr, *slot = nullptr;
     uint32_t* flags = nullptr;
     int64_t tok_cap = 0;
     int max_splits = 16;
+    int attn_chunk = -1;
     // plan (host side)
     std::vector<int32_t> cnt_h;
     int B = 0;
@@ -73,6 +78,8 @@ struct first_ctx {
     int attn_simple = -1;
     int tc_use_lo = 1;
 };
+
+constexpr int kSimpleSplitsMax = 16;
 
 namespace {
 
@@ -276,6 +283,62 @@ int launch_attn_simple(first_ctx* c, cudaStream_t st, int S, int m, const void* 
     }
 }
 
+int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorMap** out) {
+    auto it = c->kv_maps.find(ptr);
+    if (it == c->kv_maps.end() || it->second.cap_total != cap_total) {
+        first_ctx::KvMap e{};
+        e.cap_total = cap_total;
+        int rc = make_map(&e.map, ptr, (uint64_t)c->d.n_kv_heads * (uint64_t)cap_total, c->d.head_dim, attn::kTile, false);
+        if (rc) return rc;
+        it = c->kv_maps.insert_or_assign(ptr, e).first;
+    }
+    *out = &it->second.map;
+    return FIRST_OK;
+}
+
+template <int HD, int G>
+int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
+                       const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx, int C) {
+    constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_done = true;
+    }
+    FIRST_LAUNCH(kClsAttn, (attn::attn_split_mma<HD, G><<<grid, 160, smem, st>>>(
+                               tk, tv, c->q, kv->cap_total, kv->slab_off, len_l, idx, c->d.n_q_heads, C, c->o_part,
+                               c->ml_part, c->flags)));
+    return check_launch(c);
+}
+
+// Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
+int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const first_kv_cache* kv,
+                    const int32_t* len_l, const int32_t* idx, int* C_out, int* S_out) {
+    const first_model_desc& d = c->d;
+    if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
+    int C = c->attn_chunk;
+    if (C <= 0) {
+        const double est = 0.6 * (double)m * d.n_kv_heads * d.max_tokens_per_seq;
+        C = (int)(est / (8.0 * c->n_sm));
+        C = std::max(128, std::min(1024, C));
+    }
+    C = std::max(C, (d.max_tokens_per_seq + c->max_splits - 1) / c->max_splits);
+    C = (C + attn::kTile - 1) / attn::kTile * attn::kTile;
+    const int S = (d.max_tokens_per_seq + C - 1) / C;
+    const CUtensorMap *tk, *tv;
+    int rc;
+    if ((rc = kv_map_for(c, kc, kv->cap_total, &tk)) || (rc = kv_map_for(c, vc, kv->cap_total, &tv))) return rc;
+    dim3 grid(S, d.n_kv_heads, m);
+    *C_out = C;
+    *S_out = S;
+#define FIRST_ATTN_MMA(HD, G) \
+    if (d.head_dim == HD && c->group == G) return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, len_l, idx, C);
+    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
+    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
+#undef FIRST_ATTN_MMA
+    return FIRST_E_UNSUPPORTED;
+}
+
 // One projection of m compact rows: tensor cores when the row count makes it a dense
 // contraction (bf16 weights), the CUDA-core GEMV otherwise.
 //   out_mode 0: Y[j][f] = ..   (compact rows, row stride ldy)
@@ -308,7 +371,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     if ((rc = check_launch(c))) return rc;
 
     int S = (d.max_tokens_per_seq + 255) / 256;
-    S = std::max(1, std::min(S, c->max_splits));
+    S = std::max(1, std::min(S, kSimpleSplitsMax));
     const float qscale = 1.0f / std::sqrt((float)hd);
 
     for (int l = 0; l < L; ++l) {
@@ -334,9 +397,18 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                                                          static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]),
                                                          kv->cap_total, kv->slab_off, kv->slab_cap, len_l, c->flags)));
         if ((rc = check_launch(c))) return rc;
-        if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
-        FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd,
-                                                                                     t ? nullptr : c->att, xh, xl)));
+        const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
+        if (mma_attn) {
+            int Cc = 0, Sc = 0;
+            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, &Cc, &Sc))) return rc;
+            FIRST_LAUNCH(kClsAttnCombine, (attn::attn_combine_var<<<m * d.n_q_heads, 128, 0, st>>>(
+                                              c->o_part, c->ml_part, Sc, hd, d.n_q_heads, Cc, len_l, idx,
+                                              t ? nullptr : c->att, xh, xl)));
+        } else {
+            if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
+            FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd,
+                                                                                         t ? nullptr : c->att, xh, xl)));
+        }
         if ((rc = check_launch(c))) return rc;
         if ((rc = project<WT>(c, st, t, c->wo[l], t ? &c->tm_wo[l] : nullptr, D, c->qd, c->att, c->xh, c->xl, m, 1, c->x,
                               D, idx)))
@@ -437,6 +509,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
     if (cudaGetDevice(&dev) != cudaSuccess) return fail(FIRST_E_CUDA);
     cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, dev);
     const size_t MB = d.max_batch;
+    c->max_splits = std::max(kSimpleSplitsMax, std::min(64, (d.max_tokens_per_seq + 127) / 128));
     const int xw = std::max(d.d_model, c->qd);
     if ((rc = dev_alloc(&c->x, MB * d.d_model)) || (rc = dev_alloc(&c->xn, MB * xw)) ||
         (rc = dev_alloc(&c->qkv, MB * c->qkvd)) || (rc = dev_alloc(&c->q, MB * c->qd)) ||
@@ -590,6 +663,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     if (!std::strcmp(name, "max_gemv_rows")) c->max_gemv_rows = (int)value;
     else if (!std::strcmp(name, "attn_simple")) c->attn_simple = (int)value;
     else if (!std::strcmp(name, "tc_use_lo")) c->tc_use_lo = value != 0;
+    else if (!std::strcmp(name, "attn_chunk")) c->attn_chunk = (int)value;
     else return FIRST_E_ARG;
     return FIRST_OK;
 }
