@@ -296,6 +296,11 @@ def run_cuda(args, wl, shape, mask, lens):
     ms_step = ms_total / K
     value = world * B * K / (ms_total / 1e3)
 
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"quick": True, "ms_per_step": ms_step, "value": value, "layers": L,
+                              "gpu_launches": int(launches), "note": "profiling case, not a benchmark value"}))
+        return
     dense_ms, _ = timed(dense_t)
     dense_ms /= K
 
@@ -377,7 +382,8 @@ def run_cuda(args, wl, shape, mask, lens):
            "config": {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": B,
                       "prompt_lengths": [int(lens.min()), int(lens.max())], "mask": list(wl["mask"]),
                       "skip_fraction": float(1 - mask.mean()), "l2": "inputs larger than L2 (weights + KV >> 126 MB)",
-                      "parallelism": "replicas" if world > 1 else "single"},
+                      "parallelism": "replicas" if world > 1 else "single",
+                      **({"layers": L, "note": "reduced layer count: not a benchmark value"} if args.layers else {})},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
            "roofline": roof,
            "step_roofline": {"bytes_strict": bm["strict"], "bytes_full": bm["full"],
@@ -407,6 +413,10 @@ def main():
     ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-route", action="store_true")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="reduced layer count: a small case for profiler captures, never a benchmark value")
+    ap.add_argument("--quick", action="store_true",
+                    help="only the main timed loop (for profiler captures): no dense/e2e/per-kernel legs")
     args = ap.parse_args()
     wl = dict(WORKLOADS[args.workload])
     if args.mask:
@@ -416,8 +426,13 @@ def main():
         args.steps = 64 if args.impl == "cuda" else 2
     if args.impl == "reference" and args.warmup > 1:
         args.warmup = 1
-    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "cuda" and not args.quick:
+        args.warmup = max(args.warmup, 3)
     shape = SHAPES[wl["shape"]]
+    if args.layers:
+        d = shape.asdict()
+        d["n_layers"] = args.layers
+        shape = fi.ModelShape(**d)
     rank = int(os.environ.get("RANK", "0"))
     lens = fi.prompt_lengths(wl["B"], wl["lo"], wl["hi"], 1000 + rank)
     mask = make_mask(wl["mask"], wl["B"], shape.n_layers, 2000 + rank)
