@@ -232,10 +232,18 @@ int first_profile_read(first_ctx *ctx, int32_t n, double *ms, int64_t *launches,
 int32_t first_kernel_class_count(void);
 const char *first_kernel_class_name(int32_t k);
 
-/* Select kernel paths for A/B measurements.  Names: "max_gemv_rows" = largest active-row
- * count served by the CUDA-core GEMV path (rows above it use the tensor-core path when
- * the dtype is bfloat16); "attn_simple" = 1 forces the general attention kernel.  A
- * negative value restores the default.  Errors: FIRST_E_ARG for an unknown name. */
+/* Options (A/B measurements and tuning).  A negative value restores the default.
+ *   "max_gemv_rows"  largest active-row count served by the CUDA-core GEMV path; layers with
+ *                    more rows use the tensor-core path when the dtype is bfloat16 (default 2)
+ *   "attn_simple"    1 = always use the general attention kernel
+ *   "attn_chunk"     tokens per attention work item (rounded up to 64); default: from the batch
+ *   "tc_use_lo"      0 = tensor-core projections use only the bfloat16 hi half of activations
+ *   "use_graph"      0 = launch every kernel of a step directly.  Default 1: first_decode_step
+ *                    records its launch sequence once per distinct set of pointer arguments
+ *                    (tokens, outputs, cache tensors, stream) and plan, as a CUDA graph, and
+ *                    replays it; up to 8 such graphs are kept.  Nothing is captured while the
+ *                    caller's stream is itself being captured or while first_profile is on.
+ * Errors: FIRST_E_ARG for an unknown name. */
 int first_set_option(first_ctx *ctx, const char *name, int64_t value);
 
 const char *first_status_string(int status);

@@ -73,6 +73,16 @@ struct first_ctx {
     std::vector<int> ev_cls;  // class of event pair i (events 2i, 2i+1)
     double prof_ms[kNumClasses] = {};
     int64_t prof_launches[kNumClasses] = {};
+    // CUDA graphs of whole steps, keyed by every pointer the step touches and the plan version
+    struct StepGraph {
+        std::vector<const void*> key;
+        cudaGraphExec_t exec = nullptr;
+        int64_t n_launches = 0;
+        uint64_t last_use = 0;
+    };
+    std::vector<StepGraph> graphs;
+    uint64_t plan_version = 0, use_clock = 0;
+    int use_graph = 1;
     // options
     int max_gemv_rows = -1;
     int attn_simple = -1;
@@ -300,15 +310,27 @@ template <int HD, int G>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
                        const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx, int C) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_done = true;
-    }
     FIRST_LAUNCH(kClsAttn, (attn::attn_split_mma<HD, G><<<grid, 160, smem, st>>>(
                                tk, tv, c->q, kv->cap_total, kv->slab_off, len_l, idx, c->d.n_q_heads, C, c->o_part,
                                c->ml_part, c->flags)));
     return check_launch(c);
+}
+
+template <int HD, int G>
+int attn_mma_set_attr() {
+    constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
+    CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    return FIRST_OK;
+}
+
+// Opt the attention kernel of this model's (head_dim, group) into its shared-memory size (done once, at create).
+int attn_mma_setup(first_ctx* c) {
+#define FIRST_ATTN_MMA(HD, G) \
+    if (c->d.head_dim == HD && c->group == G) return attn_mma_set_attr<HD, G>();
+    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
+    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
+#undef FIRST_ATTN_MMA
+    return FIRST_OK;
 }
 
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
@@ -525,7 +547,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         if ((rc = dev_alloc(&c->xh, MB * xw)) || (rc = dev_alloc(&c->xl, MB * xw)) ||
             (rc = dev_alloc(&c->acth, MB * d.ffn_dim)) || (rc = dev_alloc(&c->actl, MB * d.ffn_dim)))
             return fail(rc);
-        if ((rc = tc_setup(c))) return fail(rc);
+        if ((rc = tc_setup(c)) || (rc = attn_mma_setup(c))) return fail(rc);
     }
     c->tok_cap = (int64_t)d.max_batch * d.max_tokens_per_seq;
     if ((rc = dev_alloc(&c->tokscore, (size_t)c->tok_cap))) return fail(rc);
@@ -545,6 +567,7 @@ int first_destroy(first_ctx* c) {
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+    for (auto& e : c->graphs) cudaGraphExecDestroy(e.exec);
     delete c;
     return FIRST_OK;
 }
@@ -614,9 +637,63 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     for (int l = 0; l < c->d.n_layers; ++l)
         if (c->cnt_h[l] > 0 && (!kv->k[l] || !kv->v[l])) return FIRST_E_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->d.dtype == FIRST_DTYPE_BF16)
-        return decode_step_impl<__nv_bfloat16>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
-    return decode_step_impl<float>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
+    auto run = [&]() {
+        if (c->d.dtype == FIRST_DTYPE_BF16)
+            return decode_step_impl<__nv_bfloat16>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
+        return decode_step_impl<float>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
+    };
+    if (!logits && next_tokens && !c->logits_int) {  // allocate outside any capture
+        int rc = dev_alloc(&c->logits_int, (size_t)c->d.max_batch * c->d.vocab);
+        if (rc) return rc;
+    }
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_TRY(cudaStreamIsCapturing(st, &cap));
+    if (!c->use_graph || c->profiling || cap != cudaStreamCaptureStatusNone) return run();
+
+    // The launch sequence of a step depends only on the plan and on the pointers: replay it as one graph.
+    std::vector<const void*> key;
+    key.reserve(12 + 2 * c->d.n_layers);
+    key.push_back(tokens); key.push_back(logits); key.push_back(next_tokens); key.push_back(layer_inputs);
+    key.push_back(kv->slab_off); key.push_back(kv->slab_cap); key.push_back(kv->len); key.push_back(kv->pos);
+    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->cap_total)));
+    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->plan_version)));
+    key.push_back(st);
+    for (int l = 0; l < c->d.n_layers; ++l) { key.push_back(kv->k[l]); key.push_back(kv->v[l]); }
+    first_ctx::StepGraph* g = nullptr;
+    for (auto& e : c->graphs)
+        if (e.key == key) { g = &e; break; }
+    if (!g) {
+        if (c->graphs.size() >= 8) {  // drop the least recently used
+            size_t lru = 0;
+            for (size_t i = 1; i < c->graphs.size(); ++i)
+                if (c->graphs[i].last_use < c->graphs[lru].last_use) lru = i;
+            cudaGraphExecDestroy(c->graphs[lru].exec);
+            c->graphs.erase(c->graphs.begin() + lru);
+        }
+        const int64_t l0 = c->launches;
+        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        const int rc = run();
+        cudaGraph_t graph = nullptr;
+        const cudaError_t e = cudaStreamEndCapture(st, &graph);
+        if (rc) {
+            if (graph) cudaGraphDestroy(graph);
+            return rc;
+        }
+        CU_TRY(e);
+        first_ctx::StepGraph sg;
+        sg.key = key;
+        sg.n_launches = c->launches - l0;
+        c->launches = l0;
+        const cudaError_t e2 = cudaGraphInstantiate(&sg.exec, graph, 0);
+        cudaGraphDestroy(graph);
+        CU_TRY(e2);
+        c->graphs.push_back(std::move(sg));
+        g = &c->graphs.back();
+    }
+    g->last_use = ++c->use_clock;
+    CU_TRY(cudaGraphLaunch(g->exec, st));
+    c->launches += g->n_launches;
+    return FIRST_OK;
 }
 
 int first_last_device_flags(first_ctx* c, uint32_t* flags, void* stream) {
@@ -664,7 +741,9 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "attn_simple")) c->attn_simple = (int)value;
     else if (!std::strcmp(name, "tc_use_lo")) c->tc_use_lo = value != 0;
     else if (!std::strcmp(name, "attn_chunk")) c->attn_chunk = (int)value;
+    else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
     else return FIRST_E_ARG;
+    c->plan_version += 1;  // cached step graphs were built under the old options
     return FIRST_OK;
 }
 
