@@ -240,7 +240,7 @@ const char *first_kernel_class_name(int32_t k);
  *   "tc_use_lo"      0 = tensor-core projections use only the bfloat16 hi half of activations
  *   "use_graph"      0 = launch every kernel of a step directly.  Default 1: first_decode_step
  *                    records its launch sequence once per distinct set of pointer arguments
- *                    (tokens, outputs, cache tensors, stream) and plan, as a CUDA graph, and
+ *                    (tokens, outputs, cache tensors) and plan, as a CUDA graph, and
  *                    replays it; up to 8 such graphs are kept.  Nothing is captured while the
  *                    caller's stream is itself being captured or while first_profile is on.
  * Errors: FIRST_E_ARG for an unknown name. */

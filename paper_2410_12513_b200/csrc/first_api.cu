@@ -82,6 +82,7 @@ struct first_ctx {
     };
     std::vector<StepGraph> graphs;
     uint64_t plan_version = 0, use_clock = 0;
+    cudaStream_t cap_stream = nullptr;  // steps are recorded here (the caller's stream may be the default one)
     int use_graph = 1;
     // options
     int max_gemv_rows = -1;
@@ -549,6 +550,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
             return fail(rc);
         if ((rc = tc_setup(c)) || (rc = attn_mma_setup(c))) return fail(rc);
     }
+    if (cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) return fail(FIRST_E_CUDA);
     c->tok_cap = (int64_t)d.max_batch * d.max_tokens_per_seq;
     if ((rc = dev_alloc(&c->tokscore, (size_t)c->tok_cap))) return fail(rc);
     std::vector<double> inv(d.head_dim / 2);
@@ -568,6 +570,7 @@ int first_destroy(first_ctx* c) {
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     for (auto& e : c->graphs) cudaGraphExecDestroy(e.exec);
+    if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     delete c;
     return FIRST_OK;
 }
@@ -637,10 +640,10 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     for (int l = 0; l < c->d.n_layers; ++l)
         if (c->cnt_h[l] > 0 && (!kv->k[l] || !kv->v[l])) return FIRST_E_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    auto run = [&]() {
+    auto run = [&](cudaStream_t s) {
         if (c->d.dtype == FIRST_DTYPE_BF16)
-            return decode_step_impl<__nv_bfloat16>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
-        return decode_step_impl<float>(c, tokens, kv, logits, next_tokens, layer_inputs, st);
+            return decode_step_impl<__nv_bfloat16>(c, tokens, kv, logits, next_tokens, layer_inputs, s);
+        return decode_step_impl<float>(c, tokens, kv, logits, next_tokens, layer_inputs, s);
     };
     if (!logits && next_tokens && !c->logits_int) {  // allocate outside any capture
         int rc = dev_alloc(&c->logits_int, (size_t)c->d.max_batch * c->d.vocab);
@@ -648,7 +651,7 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     }
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     CU_TRY(cudaStreamIsCapturing(st, &cap));
-    if (!c->use_graph || c->profiling || cap != cudaStreamCaptureStatusNone) return run();
+    if (!c->use_graph || c->profiling || cap != cudaStreamCaptureStatusNone) return run(st);
 
     // The launch sequence of a step depends only on the plan and on the pointers: replay it as one graph.
     std::vector<const void*> key;
@@ -657,7 +660,6 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     key.push_back(kv->slab_off); key.push_back(kv->slab_cap); key.push_back(kv->len); key.push_back(kv->pos);
     key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->cap_total)));
     key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->plan_version)));
-    key.push_back(st);
     for (int l = 0; l < c->d.n_layers; ++l) { key.push_back(kv->k[l]); key.push_back(kv->v[l]); }
     first_ctx::StepGraph* g = nullptr;
     for (auto& e : c->graphs)
@@ -671,10 +673,10 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
             c->graphs.erase(c->graphs.begin() + lru);
         }
         const int64_t l0 = c->launches;
-        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        const int rc = run();
+        CU_TRY(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
+        const int rc = run(c->cap_stream);
         cudaGraph_t graph = nullptr;
-        const cudaError_t e = cudaStreamEndCapture(st, &graph);
+        const cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
         if (rc) {
             if (graph) cudaGraphDestroy(graph);
             return rc;
