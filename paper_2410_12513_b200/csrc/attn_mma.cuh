@@ -9,7 +9,9 @@
 // into bfloat16 hi + lo; hi sits in rows 0..7 and lo in rows 8..15 of the same A fragment,
 // so one MMA yields both partial products and the thread adds them -- float32-grade q and p
 // against the stored bfloat16 keys/values.  Softmax is online, row maxima by quad shuffles.
-// The token axis is split in chunks of C tokens per CTA; attn_combine_var merges them.
+// The token axis is split in chunks of C tokens per CTA; the CTA that finishes a (row, kv head)
+// last (an atomic ticket) merges the chunks and writes the attention output, so no second
+// kernel is needed.
 #pragma once
 #include "common.cuh"
 #include "first.h"
@@ -46,17 +48,24 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 __device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // grid (S_max, Hkv, m), 160 threads.  Work item = (active row i, kv head h, chunk c):
-// tokens [c*C, min(T, (c+1)*C)), T = len[b] (new token already appended).  Chunks past T exit.
+// tokens [c*C, min(T, (c+1)*C)), T = len[b]+1 (the new token was just written at row len[b];
+// T = len[b] if the slab was full and nothing was written).  Chunks past T exit at once.
 // q: [m][Hq][HD] float32, pre-scaled by 1/sqrt(HD).  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64x64.
-// o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum).
+// Scratch: o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum),
+// ticket [m][Hkv] (zero between launches: the merging CTA resets it).
+// Output: out [m][Hq*HD] float32 and/or its bfloat16 hi/lo split (either may be NULL).
 template <int HD, int G>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
                                                       const float* __restrict__ q, int64_t cap_total,
                                                       const int64_t* __restrict__ slab_off,
                                                       const int32_t* __restrict__ len_l,
+                                                      const int32_t* __restrict__ slab_cap,
                                                       const int32_t* __restrict__ idx, int Hq, int C,
                                                       float* __restrict__ o_part, float2* __restrict__ ml_part,
+                                                      uint32_t* __restrict__ ticket, float* __restrict__ out,
+                                                      __nv_bfloat16* __restrict__ out_hi,
+                                                      __nv_bfloat16* __restrict__ out_lo,
                                                       uint32_t* __restrict__ flags) {
     constexpr int kHalves = HD / 64;              // 128-byte column groups per row
     constexpr int kBox = kTile * 128;             // bytes of one 64-token x 64-element box
@@ -64,11 +73,14 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     constexpr int kKSteps = HD / 16, kNTiles = HD / 8;
     static_assert(G <= 8, "query heads of a group are the 8 hi rows of the A fragment");
 
+    pdl_trigger();
+    pdl_wait();
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     const int b = idx[i];
-    const int T = len_l[b];
+    const int T = min(len_l[b] + 1, slab_cap[b]);
     const int t_begin = c * C;
     if (t_begin >= T) return;
+    const int n_chunks = (T + C - 1) / C;
     const int t_end = min(T, t_begin + C);
     const int n_tiles = (t_end - t_begin + kTile - 1) / kTile;
 
@@ -77,6 +89,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     uint8_t* base_ptr = smem_raw + (base - tc::smem_u32(smem_raw));
     __shared__ uint64_t bar_mem[2 * kStages];
     __shared__ int abort_s;
+    __shared__ int last_s;
     auto full_bar = [&](int s) { return tc::smem_u32(&bar_mem[s]); };
     auto empty_bar = [&](int s) { return tc::smem_u32(&bar_mem[kStages + s]); };
 
@@ -231,6 +244,15 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     }
     bar_consumers();
     if (!ok || abort_s) return;
+    const size_t hq0 = (size_t)i * Hq + (size_t)h * G;
+    auto emit = [&](size_t hq, int d, float y) {
+        if (out) out[hq * HD + d] = y;
+        if (out_hi) {
+            const __nv_bfloat16 hh = __float2bfloat16_rn(y);
+            out_hi[hq * HD + d] = hh;
+            out_lo[hq * HD + d] = __float2bfloat16_rn(y - __bfloat162float(hh));
+        }
+    };
     for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
         const int gg = e / HD, d = e - gg * HD;
         const float M = fmaxf(fmaxf(m_s[gg], m_s[G + gg]), fmaxf(m_s[2 * G + gg], m_s[3 * G + gg]));
@@ -244,43 +266,38 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                 l += l_s[w * G + gg] * f;
             }
         }
-        const size_t hq = (size_t)i * Hq + (size_t)h * G + gg;
-        o_part[(hq * S_max + c) * HD + d] = acc;
-        if (d == 0) ml_part[hq * S_max + c] = make_float2(M, l);
-    }
-}
-
-// Merge the chunks of each (row, query head); the number of chunks follows from the row's length.
-// out (float32) and/or its bfloat16 hi/lo split, [m][Hq*HD].
-__global__ void __launch_bounds__(128) attn_combine_var(const float* __restrict__ o_part,
-                                                        const float2* __restrict__ ml_part, int S_max, int HD, int Hq,
-                                                        int C, const int32_t* __restrict__ len_l,
-                                                        const int32_t* __restrict__ idx, float* __restrict__ out,
-                                                        __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
-    const size_t hq = blockIdx.x;
-    const int i = (int)(hq / Hq);
-    const int T = len_l[idx[i]];
-    const int S = min(S_max, (T + C - 1) / C);
-    float M = -INFINITY;
-    for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[hq * S_max + s].x);
-    float den = 0.f;
-    for (int s = 0; s < S; ++s) {
-        const float2 ml = ml_part[hq * S_max + s];
-        if (ml.x > -INFINITY) den += ml.y * __expf(ml.x - M);
-    }
-    for (int d = threadIdx.x; d < HD; d += blockDim.x) {
-        float o = 0.f;
-        for (int s = 0; s < S; ++s) {
-            const float mx = ml_part[hq * S_max + s].x;
-            if (mx > -INFINITY) o += o_part[(hq * S_max + s) * HD + d] * __expf(mx - M);
+        if (n_chunks == 1) {
+            emit(hq0 + gg, d, acc / l);  // the whole row in one chunk: done
+        } else {
+            o_part[((hq0 + gg) * S_max + c) * HD + d] = acc;
+            if (d == 0) ml_part[(hq0 + gg) * S_max + c] = make_float2(M, l);
         }
-        const float y = o / den;
-        if (out) out[hq * HD + d] = y;
-        if (hi) {
-            const __nv_bfloat16 hh = __float2bfloat16_rn(y);
-            hi[hq * HD + d] = hh;
-            lo[hq * HD + d] = __float2bfloat16_rn(y - __bfloat162float(hh));
+    }
+    if (n_chunks == 1) return;
+    // ---- ticket: the last chunk of this (row, kv head) to get here merges them all
+    __threadfence();
+    bar_consumers();
+    if (threadIdx.x == 0) {
+        const uint32_t t = atomicAdd(&ticket[(size_t)i * gridDim.y + h], 1u);
+        last_s = (t == (uint32_t)n_chunks - 1u);
+        if (last_s) ticket[(size_t)i * gridDim.y + h] = 0u;
+    }
+    bar_consumers();
+    if (!last_s) return;
+    __threadfence();
+    for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
+        const int gg = e / HD, d = e - gg * HD;
+        const size_t hq = hq0 + gg;
+        float M = -INFINITY;
+        for (int sidx = 0; sidx < n_chunks; ++sidx) M = fmaxf(M, __ldcg(&ml_part[hq * S_max + sidx].x));
+        float acc = 0.f, den = 0.f;
+        for (int sidx = 0; sidx < n_chunks; ++sidx) {
+            const float2 ml = __ldcg(&ml_part[hq * S_max + sidx]);
+            const float f = __expf(ml.x - M);
+            den += ml.y * f;
+            acc += __ldcg(&o_part[(hq * S_max + sidx) * HD + d]) * f;
         }
+        emit(hq, d, acc / den);
     }
 }
 

@@ -8,19 +8,22 @@
 namespace first {
 
 // grid (S, Hkv, m), 128 threads.  Work item = (active row i, kv head h, split s): tokens
-// [s*C, min(T,(s+1)*C)) with C = ceil(T/S), T = len[b] (the new token is already appended).
+// [s*C, min(T,(s+1)*C)) with C = ceil(T/S), T = len[b]+1 (the new token is already written at row len[b]).
 // q: [m][Hq][HD] float32, pre-scaled.  Partials: o_part [m][Hq][S][HD], ml_part [m][Hq][S] = (max, sum).
 template <typename KT, int HD, int G>
 __global__ void __launch_bounds__(128) attn_split_simple(const float* __restrict__ q, const KT* __restrict__ kc,
                                                          const KT* __restrict__ vc, int64_t cap_total,
                                                          const int64_t* __restrict__ slab_off,
                                                          const int32_t* __restrict__ len_l,
+                                                         const int32_t* __restrict__ slab_cap,
                                                          const int32_t* __restrict__ idx, int Hq,
                                                          float* __restrict__ o_part, float2* __restrict__ ml_part) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int EPL = HD / 32;
     const int S = gridDim.x, s = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     const int b = idx[i];
-    const int T = len_l[b];
+    const int T = min(len_l[b] + 1, slab_cap[b]);  // the new token sits at row len (len itself advances later)
     const int C = (T + S - 1) / S;
     const int t0 = s * C, t1 = min(T, t0 + C);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -94,6 +97,8 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* __restrict
 __global__ void __launch_bounds__(128) attn_combine(const float* __restrict__ o_part, const float2* __restrict__ ml_part,
                                                     int S, int HD, float* __restrict__ out,
                                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    pdl_trigger();
+    pdl_wait();
     const size_t hq = blockIdx.x;  // flat (row, query head)
     float M = -INFINITY;
     for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[hq * S + s].x);

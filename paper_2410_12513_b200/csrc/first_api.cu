@@ -58,7 +58,7 @@ struct first_ctx {
     float2 *ml_part = nullptr, *cs = nullptr;
     double* inv_freq = nullptr;
     int32_t *idx = nullptr, *cnt = nullptr, *slot = nullptr;
-    uint32_t* flags = nullptr;
+    uint32_t *flags = nullptr, *ticket = nullptr;
     int64_t tok_cap = 0;
     int max_splits = 16;
     int attn_chunk = -1;
@@ -84,6 +84,8 @@ struct first_ctx {
     uint64_t plan_version = 0, use_clock = 0;
     cudaStream_t cap_stream = nullptr;  // steps are recorded here (the caller's stream may be the default one)
     int use_graph = 1;
+    int use_pdl = 1;
+    bool pdl_next = false;  // the next kernel launch may overlap its predecessor (programmatic dependent launch)
     // options
     int max_gemv_rows = -1;
     int attn_simple = -1;
@@ -129,6 +131,28 @@ struct Launch {
         __VA_ARGS__;                \
     } while (0)
 
+// Launch through cudaLaunchKernelEx so that, inside a step, each kernel may start while its
+// predecessor drains (programmatic stream serialization); kernels call griddepcontrol.wait
+// before touching anything the predecessor produces.
+template <typename... P, typename... A>
+int launch_k(first_ctx* c, cudaStream_t st, int cls, void (*kern)(P...), dim3 grid, dim3 block, size_t smem,
+             A&&... args) {
+    Launch guard(c, st, cls);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = (c->use_pdl && !c->profiling && c->pdl_next) ? 1 : 0;
+    c->pdl_next = true;
+    CU_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...));
+    return FIRST_OK;
+}
+
 int check_launch(first_ctx*) {
     CU_TRY(cudaGetLastError());
     return FIRST_OK;
@@ -171,12 +195,19 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
 
 constexpr int kTcSmemMax = 210 * 1024;
 
+int tc_ksplit(const first_ctx* c, int n_out, int K, int epi) {
+    if (epi == tc::kEpiStore) return 1;
+    const int tiles = (n_out + tc::kBlockM - 1) / tc::kBlockM, kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+    const int ks = (2 * c->n_sm + tiles / 2) / tiles;
+    return std::max(1, std::min(ks, kblocks / 4));
+}
+
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
 //   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
 //   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
 int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_out, int K,
                    const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
-                   const int32_t* idx) {
+                   const int32_t* idx, bool pre_zeroed) {
     int rc;
     for (int r0 = 0; r0 < m; r0 += 256) {
         const int mm = std::min(256, m - r0);
@@ -186,12 +217,7 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
         p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
         p.use_lo = c->tc_use_lo ? 1 : 0;
         const int tiles = (n_out + tc::kBlockM - 1) / tc::kBlockM;
-        int ksplit = 1;
-        if (epi != tc::kEpiStore) {
-            ksplit = (2 * c->n_sm + tiles / 2) / tiles;
-            ksplit = std::max(1, std::min(ksplit, p.kblocks / 4));
-        }
-        p.ksplit = std::max(1, ksplit);
+        p.ksplit = tc_ksplit(c, n_out, K, epi);
         const int stage_bytes = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
         const int budget = (3 * stage_bytes <= 110 * 1024) ? 110 * 1024 : 200 * 1024;
         p.stages = std::max(1, std::min(8, budget / stage_bytes));
@@ -209,17 +235,16 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
         int e = epi;
         if (e == tc::kEpiAtomic) {
             if (p.ksplit == 1) e = tc::kEpiStore;
-            else CU_TRY(cudaMemsetAsync(p.Y, 0, (size_t)mm * ldy * sizeof(float), st));
+            else if (!pre_zeroed) {
+                CU_TRY(cudaMemsetAsync(p.Y, 0, (size_t)mm * ldy * sizeof(float), st));
+                c->pdl_next = false;
+            }
         }
         const int grid = tiles * p.ksplit;
-        if (e == tc::kEpiStore)
-            FIRST_LAUNCH(kClsGemmTc, (tc::gemm_tc_kernel<tc::kEpiStore><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
-        else if (e == tc::kEpiAtomic)
-            FIRST_LAUNCH(kClsGemmTc, (tc::gemm_tc_kernel<tc::kEpiAtomic><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
-        else
-            FIRST_LAUNCH(kClsGemmTc,
-                         (tc::gemm_tc_kernel<tc::kEpiScatterAtomic><<<grid, 192, smem, st>>>(tmA, tmBh, tmBl, p)));
-        if ((rc = check_launch(c))) return rc;
+        auto kern = e == tc::kEpiStore ? tc::gemm_tc_kernel<tc::kEpiStore>
+                    : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
+                                          : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
+        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(192), smem, tmA, tmBh, tmBl, p))) return rc;
     }
     return FIRST_OK;
 }
@@ -251,11 +276,9 @@ int launch_gemv(first_ctx* c, cudaStream_t st, const void* W, int n_out, int K, 
     for (int r0 = 0; r0 < m; r0 += 8) {
         const int rv = std::min(8, m - r0);
         const WT* w = static_cast<const WT*>(W);
-        if (rv == 1) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 1, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
-        else if (rv == 2) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 2, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
-        else if (rv <= 4) FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 4, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
-        else FIRST_LAUNCH(kClsGemv, (gemv_rows<WT, 8, EPI><<<blocks, 256, 0, st>>>(w, n_out, K, X, r0, rv, Y, ldy, idx)));
-        int rc = check_launch(c);
+        auto kern = rv == 1 ? gemv_rows<WT, 1, EPI> : rv == 2 ? gemv_rows<WT, 2, EPI>
+                    : rv <= 4 ? gemv_rows<WT, 4, EPI> : gemv_rows<WT, 8, EPI>;
+        int rc = launch_k(c, st, kClsGemv, kern, dim3(blocks), dim3(256), 0, w, n_out, K, X, r0, rv, Y, ldy, idx);
         if (rc) return rc;
     }
     return FIRST_OK;
@@ -265,12 +288,11 @@ template <typename KT, int HD>
 int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* kc, const KT* vc,
                          const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx) {
     dim3 grid(S, c->d.n_kv_heads, m);
-#define FIRST_ATTN_CASE(G)                                                                                   \
-    case G:                                                                                                  \
-        FIRST_LAUNCH(kClsAttn, (attn_split_simple<KT, HD, G><<<grid, 128, 0, st>>>(                          \
-                                   c->q, kc, vc, kv->cap_total, kv->slab_off, len_l, idx, c->d.n_q_heads,    \
-                                   c->o_part, c->ml_part)));                                                 \
-        break;
+#define FIRST_ATTN_CASE(G)                                                                                  \
+    case G:                                                                                                 \
+        return launch_k(c, st, kClsAttn, attn_split_simple<KT, HD, G>, grid, dim3(128), 0, c->q, kc, vc,    \
+                        kv->cap_total, kv->slab_off, len_l, kv->slab_cap, idx, c->d.n_q_heads, c->o_part,   \
+                        c->ml_part);
     switch (c->group) {
         FIRST_ATTN_CASE(1)
         FIRST_ATTN_CASE(2)
@@ -309,12 +331,12 @@ int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorM
 
 template <int HD, int G>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
-                       const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx, int C) {
+                       const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx, int C, float* out,
+                       __nv_bfloat16* out_hi, __nv_bfloat16* out_lo) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
-    FIRST_LAUNCH(kClsAttn, (attn::attn_split_mma<HD, G><<<grid, 160, smem, st>>>(
-                               tk, tv, c->q, kv->cap_total, kv->slab_off, len_l, idx, c->d.n_q_heads, C, c->o_part,
-                               c->ml_part, c->flags)));
-    return check_launch(c);
+    return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
+                    kv->slab_off, len_l, kv->slab_cap, idx, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
+                    out_hi, out_lo, c->flags);
 }
 
 template <int HD, int G>
@@ -336,7 +358,8 @@ int attn_mma_setup(first_ctx* c) {
 
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const first_kv_cache* kv,
-                    const int32_t* len_l, const int32_t* idx, int* C_out, int* S_out) {
+                    const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
+                    __nv_bfloat16* out_lo) {
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -352,10 +375,9 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     int rc;
     if ((rc = kv_map_for(c, kc, kv->cap_total, &tk)) || (rc = kv_map_for(c, vc, kv->cap_total, &tv))) return rc;
     dim3 grid(S, d.n_kv_heads, m);
-    *C_out = C;
-    *S_out = S;
-#define FIRST_ATTN_MMA(HD, G) \
-    if (d.head_dim == HD && c->group == G) return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, len_l, idx, C);
+#define FIRST_ATTN_MMA(HD, G)                 \
+    if (d.head_dim == HD && c->group == G)    \
+        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, len_l, idx, C, out, out_hi, out_lo);
     FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
     FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
@@ -369,10 +391,10 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
 template <typename WT>
 int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUtensorMap* tm, int n_out, int K,
             const float* X, const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int out_mode, float* Y,
-            int64_t ldy, const int32_t* idx, bool allow_split = true) {
+            int64_t ldy, const int32_t* idx, bool allow_split = true, bool pre_zeroed = false) {
     if (use_tc) {
         const int epi = out_mode == 1 ? tc::kEpiScatterAtomic : (allow_split ? tc::kEpiAtomic : tc::kEpiStore);
-        return launch_gemm_tc(c, st, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx);
+        return launch_gemm_tc(c, st, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed);
     }
     if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx);
     return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
@@ -388,19 +410,22 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 2;
     auto tc_for = [&](int m) { return kBf16 && c->tc_ready && m > gemv_max; };
     int rc;
-    FIRST_LAUNCH(kClsStepBegin, (step_begin<WT><<<B, 256, 0, st>>>(tokens, static_cast<const WT*>(c->embed), D, V,
-                                                                   kv->pos, c->inv_freq, hd / 2, c->x, c->cs,
-                                                                   c->flags)));
-    if ((rc = check_launch(c))) return rc;
+    c->pdl_next = false;  // the first kernel of a step has no predecessor to overlap
+    if ((rc = launch_k(c, st, kClsStepBegin, step_begin<WT>, dim3(B), dim3(256), 0, tokens,
+                       static_cast<const WT*>(c->embed), D, V, kv->pos, c->inv_freq, hd / 2, c->x, c->cs, c->flags)))
+        return rc;
 
     int S = (d.max_tokens_per_seq + 255) / 256;
     S = std::max(1, std::min(S, kSimpleSplitsMax));
     const float qscale = 1.0f / std::sqrt((float)hd);
+    const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
 
     for (int l = 0; l < L; ++l) {
-        if (layer_inputs)
+        if (layer_inputs) {
             CU_TRY(cudaMemcpyAsync(layer_inputs + (size_t)l * B * D, c->x, (size_t)B * D * sizeof(float),
                                    cudaMemcpyDeviceToDevice, st));
+            c->pdl_next = false;
+        }
         const int m = c->cnt_h[l];
         if (m == 0) continue;  // every sequence skips this layer: no launch at all
         const bool t = tc_for(m);
@@ -408,66 +433,59 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         int32_t* len_l = kv->len + (size_t)l * B;
         float* f32 = t ? nullptr : c->xn;
         __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
-        // attention half
-        FIRST_LAUNCH(kClsRmsnorm,
-                     (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->attn_norm[l], d.rms_eps, f32, xh, xl)));
-        if ((rc = check_launch(c))) return rc;
-        if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
-                              c->qkv, c->qkvd, nullptr)))
+        // split-K projections reduce into float32 accumulators that the preceding norm kernel clears
+        const bool zero_qkv = t && tc_ksplit(c, c->qkvd, D, tc::kEpiAtomic) > 1;
+        const bool zero_gu = t && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic) > 1;
+        // ---- attention half
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->attn_norm[l],
+                           d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))
             return rc;
-        FIRST_LAUNCH(kClsRopeAppend,
-                     (rope_append<WT><<<m, 256, 0, st>>>(c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
-                                                         static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]),
-                                                         kv->cap_total, kv->slab_off, kv->slab_cap, len_l, c->flags)));
-        if ((rc = check_launch(c))) return rc;
-        const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
+        if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
+                              c->qkv, c->qkvd, nullptr, true, zero_qkv)))
+            return rc;
+        if ((rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
+                           0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
+                           static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total, kv->slab_off,
+                           kv->slab_cap, len_l, c->flags)))
+            return rc;
         if (mma_attn) {
-            int Cc = 0, Sc = 0;
-            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, &Cc, &Sc))) return rc;
-            FIRST_LAUNCH(kClsAttnCombine, (attn::attn_combine_var<<<m * d.n_q_heads, 128, 0, st>>>(
-                                              c->o_part, c->ml_part, Sc, hd, d.n_q_heads, Cc, len_l, idx,
-                                              t ? nullptr : c->att, xh, xl)));
+            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, t ? nullptr : c->att, xh, xl)))
+                return rc;
         } else {
             if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
-            FIRST_LAUNCH(kClsAttnCombine, (attn_combine<<<m * d.n_q_heads, 128, 0, st>>>(c->o_part, c->ml_part, S, hd,
-                                                                                         t ? nullptr : c->att, xh, xl)));
+            if ((rc = launch_k(c, st, kClsAttnCombine, attn_combine, dim3(m * d.n_q_heads), dim3(128), 0, c->o_part,
+                               c->ml_part, S, hd, t ? nullptr : c->att, xh, xl)))
+                return rc;
         }
-        if ((rc = check_launch(c))) return rc;
         if ((rc = project<WT>(c, st, t, c->wo[l], t ? &c->tm_wo[l] : nullptr, D, c->qd, c->att, c->xh, c->xl, m, 1, c->x,
                               D, idx)))
             return rc;
-        // feed-forward half
-        FIRST_LAUNCH(kClsRmsnorm,
-                     (rmsnorm_rows<<<m, 256, 0, st>>>(c->x, idx, D, c->ffn_norm[l], d.rms_eps, f32, xh, xl)));
-        if ((rc = check_launch(c))) return rc;
-        if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl, m,
-                              0, c->gu, 2 * F, nullptr)))
+        // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->ffn_norm[l],
+                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap)))
             return rc;
-        FIRST_LAUNCH(kClsSiluMul, (silu_mul<<<std::min((m * F + 255) / 256, c->n_sm * 8), 256, 0, st>>>(
-                                      c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr,
-                                      t ? c->actl : nullptr)));
-        if ((rc = check_launch(c))) return rc;
+        if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl, m,
+                              0, c->gu, 2 * F, nullptr, true, zero_gu)))
+            return rc;
+        if ((rc = launch_k(c, st, kClsSiluMul, silu_mul, dim3(std::min((m * F + 255) / 256, c->n_sm * 8)), dim3(256), 0,
+                           c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr, t ? c->actl : nullptr)))
+            return rc;
         if ((rc = project<WT>(c, st, t, c->w_down[l], t ? &c->tm_wd[l] : nullptr, D, F, c->act, c->acth, c->actl, m, 1,
                               c->x, D, idx)))
             return rc;
     }
-    float* lg = logits;
-    if (!lg && next_tokens) {
-        if (!c->logits_int && (rc = dev_alloc(&c->logits_int, (size_t)d.max_batch * V))) return rc;
-        lg = c->logits_int;
-    }
+    float* lg = logits ? logits : (next_tokens ? c->logits_int : nullptr);
     if (lg) {
         const bool t = tc_for(B);
-        FIRST_LAUNCH(kClsRmsnorm, (rmsnorm_rows<<<B, 256, 0, st>>>(c->x, nullptr, D, c->final_norm, d.rms_eps,
-                                                                   t ? nullptr : c->xn, t ? c->xh : nullptr,
-                                                                   t ? c->xl : nullptr)));
-        if ((rc = check_launch(c))) return rc;
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(256), 0, c->x, nullptr, D, c->final_norm,
+                           d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
+                           nullptr)))
+            return rc;
         if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
                               nullptr, false)))
             return rc;
     }
-    FIRST_LAUNCH(kClsStepEnd, (step_end<<<B, 256, 0, st>>>(lg, V, next_tokens, kv->pos)));
-    return check_launch(c);
+    return launch_k(c, st, kClsStepEnd, step_end, dim3(B), dim3(1024), 0, lg, V, next_tokens, kv->pos);
 }
 
 }  // namespace
@@ -542,8 +560,10 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         (rc = dev_alloc(&c->ml_part, MB * d.n_q_heads * c->max_splits)) ||
         (rc = dev_alloc(&c->cs, MB * (d.head_dim / 2))) || (rc = dev_alloc(&c->inv_freq, (size_t)d.head_dim / 2)) ||
         (rc = dev_alloc(&c->idx, MB * d.n_layers)) || (rc = dev_alloc(&c->cnt, (size_t)d.n_layers)) ||
-        (rc = dev_alloc(&c->slot, MB * d.n_layers)) || (rc = dev_alloc(&c->flags, (size_t)1)))
+        (rc = dev_alloc(&c->slot, MB * d.n_layers)) || (rc = dev_alloc(&c->flags, (size_t)1)) ||
+        (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)))
         return fail(rc);
+    if (cudaMemset(c->ticket, 0, MB * d.n_kv_heads * sizeof(uint32_t)) != cudaSuccess) return fail(FIRST_E_CUDA);
     if (d.dtype == FIRST_DTYPE_BF16) {
         if ((rc = dev_alloc(&c->xh, MB * xw)) || (rc = dev_alloc(&c->xl, MB * xw)) ||
             (rc = dev_alloc(&c->acth, MB * d.ffn_dim)) || (rc = dev_alloc(&c->actl, MB * d.ffn_dim)))
@@ -565,7 +585,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
 int first_destroy(first_ctx* c) {
     if (!c) return FIRST_OK;
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
-                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl};
+                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -744,6 +764,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc_use_lo")) c->tc_use_lo = value != 0;
     else if (!std::strcmp(name, "attn_chunk")) c->attn_chunk = (int)value;
     else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
+    else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
     else return FIRST_E_ARG;
     c->plan_version += 1;  // cached step graphs were built under the old options
     return FIRST_OK;

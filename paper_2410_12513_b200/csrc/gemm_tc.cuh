@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
+    pdl_trigger();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x / p.ksplit, split = blockIdx.x - tile * p.ksplit;
     const int kb0 = (int)((int64_t)p.kblocks * split / p.ksplit), kb1 = (int)((int64_t)p.kblocks * (split + 1) / p.ksplit);
@@ -157,8 +158,22 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             const uint32_t tx = (uint32_t)stage_bytes;
-            int issued = 0;
-            for (int i = 0; i < nkb; ++i, ++issued) {
+            // Weights do not depend on the previous kernel: fill the ring with weight tiles first,
+            // then wait for the previous kernel and add the activation tiles to the same stages.
+            const int npre = min(p.stages, nkb);
+            for (int i = 0; i < npre; ++i) {
+                mbar_expect_tx(full_bar(i), tx);
+                tma_load_2d_hint(base + (uint32_t)i * stage_bytes, &tmA, full_bar(i), (kb0 + i) * kBlockK, tile * kBlockM,
+                                 pol_stream);
+            }
+            pdl_wait();
+            for (int i = 0; i < npre; ++i) {
+                const uint32_t sa = base + (uint32_t)i * stage_bytes;
+                tma_load_2d(sa + kABytes, &tmBh, full_bar(i), (kb0 + i) * kBlockK, 0);
+                if (p.use_lo) tma_load_2d(sa + kABytes + b_bytes, &tmBl, full_bar(i), (kb0 + i) * kBlockK, 0);
+            }
+            int issued = npre;
+            for (int i = npre; i < nkb; ++i, ++issued) {
                 const int s = i % p.stages;
                 const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, &abort_s, p.flags)) break;
@@ -202,6 +217,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             umma_commit(tmem_full_bar);  // accumulator complete (arrives even after a failed wait)
         }
     } else {
+        pdl_wait();  // the epilogue reads idx and reduces into buffers the previous kernels own
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok && nkb > 0) {

@@ -17,6 +17,8 @@ template <typename WT, int R, int EPI>
 __global__ void __launch_bounds__(256) gemv_rows(const WT* __restrict__ W, int n_out, int K,
                                                  const float* __restrict__ X, int r0, int rows_valid,
                                                  float* __restrict__ Y, int64_t ldy, const int32_t* __restrict__ idx) {
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;

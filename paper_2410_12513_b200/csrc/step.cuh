@@ -15,6 +15,8 @@ __global__ void __launch_bounds__(256) step_begin(const int32_t* __restrict__ to
                                                   const double* __restrict__ inv_freq, int half,
                                                   float* __restrict__ x, float2* __restrict__ cs,
                                                   uint32_t* __restrict__ flags) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x;
     int tok = tokens[b];
     if (tok < 0 || tok >= V) {
@@ -51,12 +53,28 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 // RMSNorm of the rows a layer keeps, written compactly: out[i] = norm(x[idx[i]]) * gain.
 // Also emits the bfloat16 hi/lo split (v = hi + lo up to 2^-17 relative) that the
 // tensor-core projections consume, when asked.  One block per active row.
+// Two small jobs ride along so that they need no launch of their own:
+//   zero_row: row i of a float32 accumulator (zero_cols wide) is cleared for a split-K projection;
+//   len_inc:  the row's cache length is advanced by one (unless its slab is full) -- done here,
+//             after the layer's attention, so no attention block can see a half-updated length.
 __global__ void __launch_bounds__(256) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
                                                     const float* __restrict__ gain, float eps, float* __restrict__ out,
-                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                    float* __restrict__ zero_row, int zero_cols,
+                                                    int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[8];
     const int i = blockIdx.x;
     const int b = idx ? idx[i] : i;
+    if (len_inc && threadIdx.x == 0) {
+        const int T = len_inc[b];
+        if (T < slab_cap[b]) len_inc[b] = T + 1;
+    }
+    if (zero_row) {
+        float4* z = reinterpret_cast<float4*>(zero_row + (size_t)i * zero_cols);
+        for (int k = threadIdx.x; k < zero_cols / 4; k += 256) z[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     const float* xr = x + (size_t)b * D;
     float ss = 0.f;
     for (int k = threadIdx.x * 4; k < D; k += 1024) {
@@ -80,56 +98,56 @@ __global__ void __launch_bounds__(256) rmsnorm_rows(const float* __restrict__ x,
 }
 
 // After the QKV projection: rotate q and k at the sequence's position, scale q by
-// 1/sqrt(hd), append k and v at row len[l][b] of the sequence's slab, len += 1.
-// qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  One block per active row.
-// A full slab sets FIRST_FLAG_KV_FULL and leaves cache and len alone.
+// 1/sqrt(hd), write k and v at row len[l][b] of the sequence's slab.
+// qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  grid (Hq+2*Hkv, m): one block of
+// hd/2 threads per (row, head); thread d handles the rotary pair (d, d+hd/2).
+// len is only read here (the FFN-side rmsnorm_rows advances it once attention is done).
+// A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
-__global__ void __launch_bounds__(256) rope_append(const float* __restrict__ qkv, const int32_t* __restrict__ idx,
-                                                   int Hq, int Hkv, int hd, const float2* __restrict__ cs,
-                                                   float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
-                                                   KT* __restrict__ vc, int64_t cap_total,
-                                                   const int64_t* __restrict__ slab_off,
-                                                   const int32_t* __restrict__ slab_cap, int32_t* __restrict__ len_l,
-                                                   uint32_t* __restrict__ flags) {
-    const int i = blockIdx.x, b = idx[i];
+__global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv, const int32_t* __restrict__ idx,
+                                                  int Hq, int Hkv, int hd, const float2* __restrict__ cs,
+                                                  float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
+                                                  KT* __restrict__ vc, int64_t cap_total,
+                                                  const int64_t* __restrict__ slab_off,
+                                                  const int32_t* __restrict__ slab_cap,
+                                                  const int32_t* __restrict__ len_l, uint32_t* __restrict__ flags) {
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.y, head = blockIdx.x, d = threadIdx.x, b = idx[i];
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
-    const float* row = qkv + (size_t)i * (qd + 2 * kvd);
-    const float2* csb = cs + (size_t)b * half;
+    const float* row = qkv + (size_t)i * (qd + 2 * kvd) + (size_t)head * hd;
+    const float a = row[d], bb = row[d + half];
+    if (head < Hq) {
+        const float2 c = cs[(size_t)b * half + d];
+        float* dst = q_out + (size_t)i * qd + (size_t)head * hd;
+        dst[d] = (a * c.x - bb * c.y) * qscale;
+        dst[d + half] = (bb * c.x + a * c.y) * qscale;
+        return;
+    }
     const int T = len_l[b];
-    const bool full = T >= slab_cap[b];
-    for (int p = threadIdx.x; p < Hq * half; p += blockDim.x) {
-        const int h = p / half, d = p - h * half;
-        const float2 c = csb[d];
-        const float a = row[h * hd + d], bb = row[h * hd + d + half];
-        q_out[(size_t)i * qd + h * hd + d] = (a * c.x - bb * c.y) * qscale;
-        q_out[(size_t)i * qd + h * hd + d + half] = (bb * c.x + a * c.y) * qscale;
+    if (T >= slab_cap[b]) {
+        if (head == Hq && d == 0) atomicOr(flags, FIRST_FLAG_KV_FULL);
+        return;
     }
-    if (!full) {
-        const size_t trow = (size_t)slab_off[b] + T;
-        for (int p = threadIdx.x; p < Hkv * half; p += blockDim.x) {
-            const int h = p / half, d = p - h * half;
-            const float2 c = csb[d];
-            const float a = row[qd + h * hd + d], bb = row[qd + h * hd + d + half];
-            KT* dst = kc + ((size_t)h * cap_total + trow) * hd;
-            dst[d] = from_f32<KT>(a * c.x - bb * c.y);
-            dst[d + half] = from_f32<KT>(bb * c.x + a * c.y);
-        }
-        for (int p = threadIdx.x; p < kvd; p += blockDim.x) {
-            const int h = p / hd, d = p - h * hd;
-            vc[((size_t)h * cap_total + trow) * hd + d] = from_f32<KT>(row[qd + kvd + p]);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        if (full) atomicOr(flags, FIRST_FLAG_KV_FULL);
-        else len_l[b] = T + 1;
+    const size_t trow = (size_t)slab_off[b] + T;
+    if (head < Hq + Hkv) {
+        const float2 c = cs[(size_t)b * half + d];
+        KT* dst = kc + ((size_t)(head - Hq) * cap_total + trow) * hd;
+        dst[d] = from_f32<KT>(a * c.x - bb * c.y);
+        dst[d + half] = from_f32<KT>(bb * c.x + a * c.y);
+    } else {
+        KT* dst = vc + ((size_t)(head - Hq - Hkv) * cap_total + trow) * hd;
+        dst[d] = from_f32<KT>(a);
+        dst[d + half] = from_f32<KT>(bb);
     }
 }
 
 // act[i][f] = silu(gate) * up from gu[i] = [gate(F) | up(F)]; optional bf16 hi/lo split.
 __global__ void __launch_bounds__(256) silu_mul(const float* __restrict__ gu, int m, int F, float* __restrict__ act,
                                                 __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    pdl_trigger();
+    pdl_wait();
     const size_t n = (size_t)m * F;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
         const size_t i = e / F, f = e - i * F;
@@ -145,34 +163,50 @@ __global__ void __launch_bounds__(256) silu_mul(const float* __restrict__ gu, in
 }
 
 // End of a step: greedy next token per row (lowest index among equal maxima) and pos += 1.
-__global__ void __launch_bounds__(256) step_end(const float* __restrict__ logits, int V, int32_t* __restrict__ next,
-                                                int32_t* __restrict__ pos) {
+// One block of 1024 threads per row; 16-byte loads when the row allows it.
+__global__ void __launch_bounds__(1024) step_end(const float* __restrict__ logits, int V, int32_t* __restrict__ next,
+                                                 int32_t* __restrict__ pos) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x;
     if (next && logits) {
-        __shared__ float bv[256];
-        __shared__ int bi[256];
+        __shared__ float bv[32];
+        __shared__ int bi[32];
         const float* row = logits + (size_t)b * V;
         float best = -INFINITY;
         int besti = 0x7fffffff;
-        for (int i = threadIdx.x; i < V; i += 256) {
-            const float v = row[i];
+        auto consider = [&](float v, int i) {
             if (v > best || (v == best && i < besti)) { best = v; besti = i; }
-        }
-        bv[threadIdx.x] = best;
-        bi[threadIdx.x] = besti;
-        __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
-            if (threadIdx.x < o) {
-                const float v = bv[threadIdx.x + o];
-                const int j = bi[threadIdx.x + o];
-                if (v > bv[threadIdx.x] || (v == bv[threadIdx.x] && j < bi[threadIdx.x])) {
-                    bv[threadIdx.x] = v;
-                    bi[threadIdx.x] = j;
-                }
+        };
+        if ((V & 3) == 0) {
+            const float4* r4 = reinterpret_cast<const float4*>(row);
+#pragma unroll 4
+            for (int i = threadIdx.x; i < V / 4; i += 1024) {
+                const float4 v = r4[i];
+                consider(v.x, 4 * i); consider(v.y, 4 * i + 1); consider(v.z, 4 * i + 2); consider(v.w, 4 * i + 3);
             }
-            __syncthreads();
+        } else {
+            for (int i = threadIdx.x; i < V; i += 1024) consider(row[i], i);
         }
-        if (threadIdx.x == 0) next[b] = bi[0] == 0x7fffffff ? 0 : bi[0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v = __shfl_xor_sync(0xffffffffu, best, o);
+            const int j = __shfl_xor_sync(0xffffffffu, besti, o);
+            consider(v, j);
+        }
+        if ((threadIdx.x & 31) == 0) { bv[threadIdx.x >> 5] = best; bi[threadIdx.x >> 5] = besti; }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            best = bv[threadIdx.x];
+            besti = bi[threadIdx.x];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float v = __shfl_xor_sync(0xffffffffu, best, o);
+                const int j = __shfl_xor_sync(0xffffffffu, besti, o);
+                consider(v, j);
+            }
+            if (threadIdx.x == 0) next[b] = besti == 0x7fffffff ? 0 : besti;
+        }
     }
     if (threadIdx.x == 0) pos[b] += 1;
 }
