@@ -223,6 +223,9 @@ def run_cuda(args, wl, shape, mask, lens):
     len_t, pos_t = len0.clone(), pos0.clone()
     kv = KVCache(kk, vv, torch.from_numpy(off).to(dev), torch.from_numpy(caps).to(dev), len_t, pos_t)
     ctx = FirstContext(shape, 1, B, int(caps.max()), weights)
+    for kv_ in args.opt:
+        name, val = kv_.split("=")
+        ctx.set_option(name, int(val))
     stream = torch.cuda.current_stream()
 
     tok0 = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).to(dev)
@@ -383,6 +386,7 @@ def run_cuda(args, wl, shape, mask, lens):
                       "prompt_lengths": [int(lens.min()), int(lens.max())], "mask": list(wl["mask"]),
                       "skip_fraction": float(1 - mask.mean()), "l2": "inputs larger than L2 (weights + KV >> 126 MB)",
                       "parallelism": "replicas" if world > 1 else "single",
+                      **({"options": args.opt} if args.opt else {}),
                       **({"layers": L, "note": "reduced layer count: not a benchmark value"} if args.layers else {})},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
            "roofline": roof,
@@ -413,6 +417,7 @@ def main():
     ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-route", action="store_true")
+    ap.add_argument("--opt", action="append", default=[], help="library option name=value (A/B runs)")
     ap.add_argument("--layers", type=int, default=None,
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
     ap.add_argument("--quick", action="store_true",
