@@ -285,19 +285,39 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     bar_consumers();
     if (!last_s) return;
     __threadfence();
+    // Merge: (1) all chunk statistics into shared memory at once, (2) one weight per (head, chunk),
+    // (3) weighted sums with independent loads.  o_s is free again (everyone passed the barrier).
+    float* w_s = o_s;  // [2][G][64]
+    for (int e = threadIdx.x; e < G * n_chunks; e += kConsumers) {
+        const int gg = e / n_chunks, sidx = e - gg * n_chunks;
+        const float2 ml = __ldcg(&ml_part[(hq0 + gg) * S_max + sidx]);
+        w_s[gg * 64 + sidx] = ml.x;
+        w_s[(G + gg) * 64 + sidx] = ml.y;
+    }
+    bar_consumers();
+    if (threadIdx.x < G) {
+        const int gg = threadIdx.x;
+        float M = -INFINITY, den = 0.f;
+        for (int sidx = 0; sidx < n_chunks; ++sidx) M = fmaxf(M, w_s[gg * 64 + sidx]);
+        for (int sidx = 0; sidx < n_chunks; ++sidx) den += w_s[(G + gg) * 64 + sidx] * __expf(w_s[gg * 64 + sidx] - M);
+        const float inv = 1.f / den;
+        for (int sidx = 0; sidx < n_chunks; ++sidx) w_s[gg * 64 + sidx] = __expf(w_s[gg * 64 + sidx] - M) * inv;
+    }
+    bar_consumers();
     for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
         const int gg = e / HD, d = e - gg * HD;
         const size_t hq = hq0 + gg;
-        float M = -INFINITY;
-        for (int sidx = 0; sidx < n_chunks; ++sidx) M = fmaxf(M, __ldcg(&ml_part[hq * S_max + sidx].x));
-        float acc = 0.f, den = 0.f;
-        for (int sidx = 0; sidx < n_chunks; ++sidx) {
-            const float2 ml = __ldcg(&ml_part[hq * S_max + sidx]);
-            const float f = __expf(ml.x - M);
-            den += ml.y * f;
-            acc += __ldcg(&o_part[(hq * S_max + sidx) * HD + d]) * f;
+        const float* src = o_part + (hq * S_max) * HD + d;
+        const float* wv = w_s + gg * 64;
+        float acc = 0.f;
+        int sidx = 0;
+        for (; sidx + 4 <= n_chunks; sidx += 4) {
+            const float v0 = __ldcg(src + (size_t)(sidx + 0) * HD), v1 = __ldcg(src + (size_t)(sidx + 1) * HD);
+            const float v2 = __ldcg(src + (size_t)(sidx + 2) * HD), v3 = __ldcg(src + (size_t)(sidx + 3) * HD);
+            acc += v0 * wv[sidx] + v1 * wv[sidx + 1] + v2 * wv[sidx + 2] + v3 * wv[sidx + 3];
         }
-        emit(hq, d, acc / den);
+        for (; sidx < n_chunks; ++sidx) acc += __ldcg(src + (size_t)sidx * HD) * wv[sidx];
+        emit(hq, d, acc);
     }
 }
 
