@@ -243,6 +243,9 @@ const char *first_kernel_class_name(int32_t k);
  *                    (tokens, outputs, cache tensors) and plan, as a CUDA graph, and
  *                    replays it; up to 8 such graphs are kept.  Nothing is captured while the
  *                    caller's stream is itself being captured or while first_profile is on.
+ *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
+ *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
+ *                    its epilogue (needs ffn_dim % 64 == 0).
  *   "use_pdl"        0 = kernels of a step are launched strictly one after another.  Default 1:
  *                    programmatic dependent launch lets a kernel's prologue (and, for the
  *                    projections, its first weight tiles) overlap the previous kernel's tail.

@@ -50,7 +50,7 @@ struct first_ctx {
     float *o_part = nullptr, *logits_int = nullptr, *tokscore = nullptr;
     __nv_bfloat16 *xh = nullptr, *xl = nullptr, *acth = nullptr, *actl = nullptr;  // hi/lo activation splits
     // TMA descriptors of the weight matrices (bf16 models)
-    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wgu64, tm_wd;  // tm_wgu64: 64-row boxes (gate|up pairing)
     CUtensorMap tm_lm{};
     bool tc_ready = false;
     struct KvMap { int64_t cap_total; CUtensorMap map; };
@@ -90,6 +90,7 @@ struct first_ctx {
     int max_gemv_rows = -1;
     int attn_simple = -1;
     int tc_use_lo = 1;
+    int fuse_swiglu = 1;
 };
 
 constexpr int kSimpleSplitsMax = 16;
@@ -207,7 +208,8 @@ int tc_ksplit(const first_ctx* c, int n_out, int K, int epi) {
 //   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
 int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_out, int K,
                    const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
-                   const int32_t* idx, bool pre_zeroed) {
+                   const int32_t* idx, bool pre_zeroed, float* act = nullptr, __nv_bfloat16* act_hi = nullptr,
+                   __nv_bfloat16* act_lo = nullptr) {
     int rc;
     for (int r0 = 0; r0 < m; r0 += 256) {
         const int mm = std::min(256, m - r0);
@@ -216,15 +218,18 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
         p.n_pad = (mm + 15) / 16 * 16;
         p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
         p.use_lo = c->tc_use_lo ? 1 : 0;
-        const int tiles = (n_out + tc::kBlockM - 1) / tc::kBlockM;
-        p.ksplit = tc_ksplit(c, n_out, K, epi);
+        const int tiles = epi == tc::kEpiSwiglu ? n_out / 64 : (n_out + tc::kBlockM - 1) / tc::kBlockM;
+        p.ksplit = epi == tc::kEpiSwiglu ? 1 : tc_ksplit(c, n_out, K, epi);
+        p.act = act ? act + (size_t)r0 * n_out : nullptr;
+        p.act_hi = act_hi ? act_hi + (size_t)r0 * n_out : nullptr;
+        p.act_lo = act_lo ? act_lo + (size_t)r0 * n_out : nullptr;
         const int stage_bytes = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
         const int budget = (3 * stage_bytes <= 110 * 1024) ? 110 * 1024 : 200 * 1024;
         p.stages = std::max(1, std::min(8, budget / stage_bytes));
         int cols = 32;
         while (cols < p.n_pad) cols *= 2;
         p.tmem_cols = cols;
-        p.Y = Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy);
+        p.Y = Y ? Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy) : nullptr;
         p.ldy = ldy;
         p.idx = idx ? idx + r0 : nullptr;
         p.flags = c->flags;
@@ -243,6 +248,7 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
         const int grid = tiles * p.ksplit;
         auto kern = e == tc::kEpiStore ? tc::gemm_tc_kernel<tc::kEpiStore>
                     : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
+                    : e == tc::kEpiSwiglu ? tc::gemm_tc_kernel<tc::kEpiSwiglu>
                                           : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
         if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(192), smem, tmA, tmBh, tmBl, p))) return rc;
     }
@@ -253,11 +259,12 @@ int tc_setup(first_ctx* c) {
     const first_model_desc& d = c->d;
     int rc;
     const int L = d.n_layers;
-    c->tm_wqkv.resize(L); c->tm_wo.resize(L); c->tm_wgu.resize(L); c->tm_wd.resize(L);
+    c->tm_wqkv.resize(L); c->tm_wo.resize(L); c->tm_wgu.resize(L); c->tm_wgu64.resize(L); c->tm_wd.resize(L);
     for (int l = 0; l < L; ++l) {
         if ((rc = make_map(&c->tm_wqkv[l], c->wqkv[l], c->qkvd, d.d_model, tc::kBlockM, true)) ||
             (rc = make_map(&c->tm_wo[l], c->wo[l], d.d_model, c->qd, tc::kBlockM, true)) ||
             (rc = make_map(&c->tm_wgu[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, tc::kBlockM, true)) ||
+            (rc = make_map(&c->tm_wgu64[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, 64, true)) ||
             (rc = make_map(&c->tm_wd[l], c->w_down[l], d.d_model, d.ffn_dim, tc::kBlockM, true)))
             return rc;
     }
@@ -265,6 +272,7 @@ int tc_setup(first_ctx* c) {
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiScatterAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiSwiglu>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
     c->tc_ready = true;
     return FIRST_OK;
 }
@@ -435,7 +443,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
         // split-K projections reduce into float32 accumulators that the preceding norm kernel clears
         const bool zero_qkv = t && tc_ksplit(c, c->qkvd, D, tc::kEpiAtomic) > 1;
-        const bool zero_gu = t && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic) > 1;
+        const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
+        const bool zero_gu = t && !fused_ffn && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic) > 1;
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))
@@ -464,12 +473,20 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->ffn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap)))
             return rc;
-        if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl, m,
-                              0, c->gu, 2 * F, nullptr, true, zero_gu)))
-            return rc;
-        if ((rc = launch_k(c, st, kClsSiluMul, silu_mul, dim3(std::min((m * F + 255) / 256, c->n_sm * 8)), dim3(256), 0,
-                           c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr, t ? c->actl : nullptr)))
-            return rc;
+        if (fused_ffn) {
+            // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
+            if ((rc = launch_gemm_tc(c, st, c->tm_wgu64[l], F, D, c->xh, c->xl, m, tc::kEpiSwiglu, nullptr, 0, nullptr,
+                                     false, nullptr, c->acth, c->actl)))
+                return rc;
+        } else {
+            if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl,
+                                  m, 0, c->gu, 2 * F, nullptr, true, zero_gu)))
+                return rc;
+            if ((rc = launch_k(c, st, kClsSiluMul, silu_mul, dim3(std::min((m * F + 255) / 256, c->n_sm * 8)),
+                               dim3(256), 0, c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr,
+                               t ? c->actl : nullptr)))
+                return rc;
+        }
         if ((rc = project<WT>(c, st, t, c->w_down[l], t ? &c->tm_wd[l] : nullptr, D, F, c->act, c->acth, c->actl, m, 1,
                               c->x, D, idx)))
             return rc;
@@ -765,6 +782,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "attn_chunk")) c->attn_chunk = (int)value;
     else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
     else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
+    else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
     else return FIRST_E_ARG;
     c->plan_version += 1;  // cached step graphs were built under the old options
     return FIRST_OK;

@@ -10,6 +10,9 @@
 //
 // Work unit = (128-feature tile, K range).  With several K ranges per tile the partial sums
 // meet in global memory through float32 reductions (red.global.add).
+// The gate/up projection has its own epilogue: its tile is 64 gate rows stacked on the matching
+// 64 up rows (two TMA boxes), the whole K range in one CTA, and the epilogue applies
+// silu(gate)*up in registers and writes the activation (and its hi/lo split) directly.
 // Roles inside a CTA of 6 warps: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (one TMEM lane quadrant each).  Every wait is bounded.
 #pragma once
@@ -27,7 +30,7 @@ constexpr int kUmmaK = 16;
 constexpr int kABytes = kBlockM * kBlockK * 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-enum Epilogue { kEpiStore = 0, kEpiAtomic = 1, kEpiScatterAtomic = 2 };
+enum Epilogue { kEpiStore = 0, kEpiAtomic = 1, kEpiScatterAtomic = 2, kEpiSwiglu = 3 };
 
 struct GemmParams {
     int n_out, K, m, n_pad;
@@ -37,6 +40,11 @@ struct GemmParams {
     int64_t ldy;
     const int32_t* idx;
     uint32_t* flags;
+    // kEpiSwiglu: the weight matrix is [gate rows (n_out) | up rows (n_out)]; a tile pairs 64 gate
+    // features with the same 64 up features and the epilogue writes silu(gate)*up:
+    float* act;              // [m][n_out] float32 or NULL
+    __nv_bfloat16* act_hi;   // [m][n_out] bfloat16 hi/lo split or NULL
+    __nv_bfloat16* act_lo;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -158,13 +166,20 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             const uint32_t tx = (uint32_t)stage_bytes;
+            auto load_a = [&](uint32_t sa, uint32_t bar, int kc) {
+                if (EPI == kEpiSwiglu) {
+                    tma_load_2d_hint(sa, &tmA, bar, kc, tile * 64, pol_stream);                      // gate rows
+                    tma_load_2d_hint(sa + kABytes / 2, &tmA, bar, kc, p.n_out + tile * 64, pol_stream);  // up rows
+                } else {
+                    tma_load_2d_hint(sa, &tmA, bar, kc, tile * kBlockM, pol_stream);
+                }
+            };
             // Weights do not depend on the previous kernel: fill the ring with weight tiles first,
             // then wait for the previous kernel and add the activation tiles to the same stages.
             const int npre = min(p.stages, nkb);
             for (int i = 0; i < npre; ++i) {
                 mbar_expect_tx(full_bar(i), tx);
-                tma_load_2d_hint(base + (uint32_t)i * stage_bytes, &tmA, full_bar(i), (kb0 + i) * kBlockK, tile * kBlockM,
-                                 pol_stream);
+                load_a(base + (uint32_t)i * stage_bytes, full_bar(i), (kb0 + i) * kBlockK);
             }
             pdl_wait();
             for (int i = 0; i < npre; ++i) {
@@ -180,7 +195,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 const uint32_t sa = base + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full_bar(s), tx);
                 const int kc = (kb0 + i) * kBlockK;
-                tma_load_2d_hint(sa, &tmA, full_bar(s), kc, tile * kBlockM, pol_stream);
+                load_a(sa, full_bar(s), kc);
                 tma_load_2d(sa + kABytes, &tmBh, full_bar(s), kc, 0);
                 if (p.use_lo) tma_load_2d(sa + kABytes + b_bytes, &tmBl, full_bar(s), kc, 0);
             }
@@ -220,8 +235,52 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
         pdl_wait();  // the epilogue reads idx and reduces into buffers the previous kernels own
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok && nkb > 0) {
+        if (EPI == kEpiSwiglu) {
+            // lanes 0..63 of the accumulator hold gate features, lanes 64..127 the matching up features.
+            // Up warps park their values in shared memory (the ring is idle once the accumulator is
+            // complete), gate warps combine.  u_s[j][feature]: conflict-free both ways.
             const int quad = warp & 3;
+            float* u_s = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)));
+            const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
+            const bool run = ok && nkb > 0;
+            if (quad >= 2 && run) {
+                const int fl = (quad - 2) * 32 + lane;
+                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_addr + (uint32_t)c0, v);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) u_s[(c0 + c) * 64 + fl] = __uint_as_float(v[c]);
+                }
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (quad < 2 && run) {
+                const int fl = quad * 32 + lane;
+                const int f = tile * 64 + fl;
+                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_addr + (uint32_t)c0, v);
+                    if (f < p.n_out) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int j = c0 + c;
+                            if (j < p.m) {
+                                const float g = __uint_as_float(v[c]);
+                                const float y = g / (1.f + expf(-g)) * u_s[j * 64 + fl];
+                                const size_t o = (size_t)j * p.n_out + f;
+                                if (p.act) p.act[o] = y;
+                                if (p.act_hi) {
+                                    const __nv_bfloat16 h = __float2bfloat16_rn(y);
+                                    p.act_hi[o] = h;
+                                    p.act_lo[o] = __float2bfloat16_rn(y - __bfloat162float(h));
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        } else if (ok && nkb > 0) {
+            const int quad = warp & 3;
+
             const int f = tile * kBlockM + quad * 32 + lane;
             const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
             for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
