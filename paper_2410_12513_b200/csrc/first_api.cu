@@ -373,8 +373,8 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     int C = c->attn_chunk;
     if (C <= 0) {
         const double est = 0.6 * (double)m * d.n_kv_heads * d.max_tokens_per_seq;
-        C = (int)(est / (8.0 * c->n_sm));
-        C = std::max(128, std::min(1024, C));
+        C = (int)(est / (4.0 * c->n_sm));
+        C = std::max(512, std::min(2048, C));
     }
     C = std::max(C, (d.max_tokens_per_seq + c->max_splits - 1) / c->max_splits);
     C = (C + attn::kTile - 1) / attn::kTile * attn::kTile;
