@@ -91,6 +91,8 @@ struct first_ctx {
     int attn_simple = -1;
     int tc_use_lo = 1;
     int fuse_swiglu = 1;
+    int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
+    int tc_mt2_min_rows = 49;  // from this many active rows on, a projection CTA takes two weight tiles
 };
 
 constexpr int kSimpleSplitsMax = 16;
@@ -196,9 +198,10 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
 
 constexpr int kTcSmemMax = 210 * 1024;
 
-int tc_ksplit(const first_ctx* c, int n_out, int K, int epi) {
+int tc_ksplit(const first_ctx* c, int n_out, int K, int epi, int m) {
     if (epi == tc::kEpiStore) return 1;
-    const int tiles = (n_out + tc::kBlockM - 1) / tc::kBlockM, kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+    const int mt = (std::min(m, 256) >= c->tc_mt2_min_rows) ? 2 : 1;
+    const int tiles = (n_out + tc::kBlockM * mt - 1) / (tc::kBlockM * mt), kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
     const int ks = (2 * c->n_sm + tiles / 2) / tiles;
     return std::max(1, std::min(ks, kblocks / 4));
 }
@@ -206,7 +209,7 @@ int tc_ksplit(const first_ctx* c, int n_out, int K, int epi) {
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
 //   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
 //   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
-int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_out, int K,
+int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmA2, int n_out, int K,
                    const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
                    const int32_t* idx, bool pre_zeroed, float* act = nullptr, __nv_bfloat16* act_hi = nullptr,
                    __nv_bfloat16* act_lo = nullptr) {
@@ -218,17 +221,25 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
         p.n_pad = (mm + 15) / 16 * 16;
         p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
         p.use_lo = c->tc_use_lo ? 1 : 0;
-        const int tiles = epi == tc::kEpiSwiglu ? n_out / 64 : (n_out + tc::kBlockM - 1) / tc::kBlockM;
-        p.ksplit = epi == tc::kEpiSwiglu ? 1 : tc_ksplit(c, n_out, K, epi);
+        p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
+        if (epi == tc::kEpiSwiglu && n_out % 128) p.mt = 1;
+        const int tile_rows = (epi == tc::kEpiSwiglu ? 64 : tc::kBlockM) * p.mt;
+        const int tiles = (n_out + tile_rows - 1) / tile_rows;
+        p.ksplit = 1;
+        if (epi != tc::kEpiSwiglu && epi != tc::kEpiStore) {
+            const int ks = (2 * c->n_sm + tiles / 2) / tiles;
+            p.ksplit = std::max(1, std::min(ks, p.kblocks / 4));
+        }
         p.act = act ? act + (size_t)r0 * n_out : nullptr;
         p.act_hi = act_hi ? act_hi + (size_t)r0 * n_out : nullptr;
         p.act_lo = act_lo ? act_lo + (size_t)r0 * n_out : nullptr;
-        const int stage_bytes = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
-        const int budget = (3 * stage_bytes <= 110 * 1024) ? 110 * 1024 : 200 * 1024;
+        const int stage_bytes = tc::kABytes * p.mt + p.n_pad * 128 * (p.use_lo ? 2 : 1);
+        const int budget = (3 * stage_bytes <= c->tc_smem_kb * 1024) ? c->tc_smem_kb * 1024 : 200 * 1024;
         p.stages = std::max(1, std::min(8, budget / stage_bytes));
         int cols = 32;
         while (cols < p.n_pad) cols *= 2;
-        p.tmem_cols = cols;
+        p.acc_cols = cols;
+        p.tmem_cols = std::max(32, cols * p.mt);
         p.Y = Y ? Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy) : nullptr;
         p.ldy = ldy;
         p.idx = idx ? idx + r0 : nullptr;
@@ -250,7 +261,7 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_
                     : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
                     : e == tc::kEpiSwiglu ? tc::gemm_tc_kernel<tc::kEpiSwiglu>
                                           : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
-        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(192), smem, tmA, tmBh, tmBl, p))) return rc;
+        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(192), smem, tmA, tmA2, tmBh, tmBl, p))) return rc;
     }
     return FIRST_OK;
 }
@@ -402,7 +413,7 @@ int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUt
             int64_t ldy, const int32_t* idx, bool allow_split = true, bool pre_zeroed = false) {
     if (use_tc) {
         const int epi = out_mode == 1 ? tc::kEpiScatterAtomic : (allow_split ? tc::kEpiAtomic : tc::kEpiStore);
-        return launch_gemm_tc(c, st, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed);
+        return launch_gemm_tc(c, st, *tm, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed);
     }
     if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx);
     return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
@@ -442,9 +453,9 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         float* f32 = t ? nullptr : c->xn;
         __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
         // split-K projections reduce into float32 accumulators that the preceding norm kernel clears
-        const bool zero_qkv = t && tc_ksplit(c, c->qkvd, D, tc::kEpiAtomic) > 1;
+        const bool zero_qkv = t && tc_ksplit(c, c->qkvd, D, tc::kEpiAtomic, m) > 1;
         const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
-        const bool zero_gu = t && !fused_ffn && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic) > 1;
+        const bool zero_gu = t && !fused_ffn && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic, m) > 1;
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))
@@ -475,7 +486,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
-            if ((rc = launch_gemm_tc(c, st, c->tm_wgu64[l], F, D, c->xh, c->xl, m, tc::kEpiSwiglu, nullptr, 0, nullptr,
+            if ((rc = launch_gemm_tc(c, st, c->tm_wgu64[l], c->tm_wgu[l], F, D, c->xh, c->xl, m, tc::kEpiSwiglu, nullptr, 0, nullptr,
                                      false, nullptr, c->acth, c->actl)))
                 return rc;
         } else {
@@ -783,6 +794,8 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
     else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
+    else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : 49;
+    else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
     else return FIRST_E_ARG;
     c->plan_version += 1;  // cached step graphs were built under the old options
     return FIRST_OK;

@@ -36,6 +36,9 @@ struct GemmParams {
     int n_out, K, m, n_pad;
     int kblocks, ksplit;
     int stages, tmem_cols, use_lo;
+    int mt;        // 128-row weight tiles per CTA (1 or 2): two tiles share every activation tile, which
+                   // halves the activation bytes pulled from L2 per weight byte when there are many rows
+    int acc_cols;  // TMEM columns per accumulator (power of two >= n_pad)
     float* Y;
     int64_t ldy;
     const int32_t* idx;
@@ -120,15 +123,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Dynamic shared memory: [stages][A 16 KB | B_hi n_pad*128 | B_lo n_pad*128] (1024-aligned), then barriers.
+// Dynamic shared memory: [stages][A mt*16 KB | B_hi n_pad*128 | B_lo n_pad*128] (1024-aligned), then barriers.
 template <int EPI>
 __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                      const __grid_constant__ CUtensorMap tmA2,
                                                       const __grid_constant__ CUtensorMap tmBh,
                                                       const __grid_constant__ CUtensorMap tmBl, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int b_bytes = p.n_pad * 128;
-    const int stage_bytes = kABytes + b_bytes * (p.use_lo ? 2 : 1);
+    const int a_bytes = kABytes * p.mt;
+    const int stage_bytes = a_bytes + b_bytes * (p.use_lo ? 2 : 1);
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;  // full[S], empty[S], tmem_full : 8 B each
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (p.stages + s); };
@@ -168,10 +173,14 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             const uint32_t tx = (uint32_t)stage_bytes;
             auto load_a = [&](uint32_t sa, uint32_t bar, int kc) {
                 if (EPI == kEpiSwiglu) {
-                    tma_load_2d_hint(sa, &tmA, bar, kc, tile * 64, pol_stream);                      // gate rows
-                    tma_load_2d_hint(sa + kABytes / 2, &tmA, bar, kc, p.n_out + tile * 64, pol_stream);  // up rows
+                    // gate rows, then the matching up rows: 64+64 (mt = 1) or 128+128 (mt = 2)
+                    const int rows = 64 * p.mt;
+                    const CUtensorMap* tm = p.mt == 1 ? &tmA : &tmA2;
+                    tma_load_2d_hint(sa, tm, bar, kc, tile * rows, pol_stream);
+                    tma_load_2d_hint(sa + a_bytes / 2, tm, bar, kc, p.n_out + tile * rows, pol_stream);
                 } else {
-                    tma_load_2d_hint(sa, &tmA, bar, kc, tile * kBlockM, pol_stream);
+                    for (int a = 0; a < p.mt; ++a)
+                        tma_load_2d_hint(sa + a * kABytes, &tmA, bar, kc, (tile * p.mt + a) * kBlockM, pol_stream);
                 }
             };
             // Weights do not depend on the previous kernel: fill the ring with weight tiles first,
@@ -184,8 +193,8 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             pdl_wait();
             for (int i = 0; i < npre; ++i) {
                 const uint32_t sa = base + (uint32_t)i * stage_bytes;
-                tma_load_2d(sa + kABytes, &tmBh, full_bar(i), (kb0 + i) * kBlockK, 0);
-                if (p.use_lo) tma_load_2d(sa + kABytes + b_bytes, &tmBl, full_bar(i), (kb0 + i) * kBlockK, 0);
+                tma_load_2d(sa + a_bytes, &tmBh, full_bar(i), (kb0 + i) * kBlockK, 0);
+                if (p.use_lo) tma_load_2d(sa + a_bytes + b_bytes, &tmBl, full_bar(i), (kb0 + i) * kBlockK, 0);
             }
             int issued = npre;
             for (int i = npre; i < nkb; ++i, ++issued) {
@@ -196,8 +205,8 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 mbar_expect_tx(full_bar(s), tx);
                 const int kc = (kb0 + i) * kBlockK;
                 load_a(sa, full_bar(s), kc);
-                tma_load_2d(sa + kABytes, &tmBh, full_bar(s), kc, 0);
-                if (p.use_lo) tma_load_2d(sa + kABytes + b_bytes, &tmBl, full_bar(s), kc, 0);
+                tma_load_2d(sa + a_bytes, &tmBh, full_bar(s), kc, 0);
+                if (p.use_lo) tma_load_2d(sa + a_bytes + b_bytes, &tmBl, full_bar(s), kc, 0);
             }
             if (abort_s) {
                 // let the copies already issued land before this CTA's shared memory goes away
@@ -218,14 +227,17 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                const uint64_t da = smem_desc_sw128(sa), dbh = smem_desc_sw128(sa + kABytes);
+                const uint64_t dbh = smem_desc_sw128(sa + a_bytes), dbl = smem_desc_sw128(sa + a_bytes + b_bytes);
+                for (int a = 0; a < p.mt; ++a) {
+                    const uint64_t da = smem_desc_sw128(sa + a * kABytes);
+                    const uint32_t td = tmem_d + (uint32_t)(a * p.acc_cols);
 #pragma unroll
-                for (int k = 0; k < kBlockK / kUmmaK; ++k)
-                    umma_bf16(tmem_d, da + 2u * k, dbh + 2u * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                if (p.use_lo) {
-                    const uint64_t dbl = smem_desc_sw128(sa + kABytes + b_bytes);
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                        umma_bf16(td, da + 2u * k, dbh + 2u * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    if (p.use_lo) {
 #pragma unroll
-                    for (int k = 0; k < kBlockK / kUmmaK; ++k) umma_bf16(tmem_d, da + 2u * k, dbl + 2u * k, idesc, 1u);
+                        for (int k = 0; k < kBlockK / kUmmaK; ++k) umma_bf16(td, da + 2u * k, dbl + 2u * k, idesc, 1u);
+                    }
                 }
                 umma_commit(empty_bar(s));  // frees the stage once these MMAs have read it
             }
@@ -235,7 +247,36 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
         pdl_wait();  // the epilogue reads idx and reduces into buffers the previous kernels own
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (EPI == kEpiSwiglu) {
+        if (EPI == kEpiSwiglu && p.mt == 2) {
+            // accumulator 0 = 128 gate features, accumulator 1 = the same 128 up features: no exchange needed
+            const int quad = warp & 3;
+            const int f = tile * 128 + quad * 32 + lane;
+            const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
+            if (ok && nkb > 0) {
+                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    uint32_t vg[16], vu[16];
+                    tmem_ld16(lane_addr + (uint32_t)c0, vg);
+                    tmem_ld16(lane_addr + (uint32_t)(p.acc_cols + c0), vu);
+                    if (f < p.n_out) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int j = c0 + c;
+                            if (j < p.m) {
+                                const float g = __uint_as_float(vg[c]);
+                                const float y = g / (1.f + expf(-g)) * __uint_as_float(vu[c]);
+                                const size_t o = (size_t)j * p.n_out + f;
+                                if (p.act) p.act[o] = y;
+                                if (p.act_hi) {
+                                    const __nv_bfloat16 h = __float2bfloat16_rn(y);
+                                    p.act_hi[o] = h;
+                                    p.act_lo[o] = __float2bfloat16_rn(y - __bfloat162float(h));
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        } else if (EPI == kEpiSwiglu) {
             // lanes 0..63 of the accumulator hold gate features, lanes 64..127 the matching up features.
             // Up warps park their values in shared memory (the ring is idle once the accumulator is
             // complete), gate warps combine.  u_s[j][feature]: conflict-free both ways.
@@ -280,21 +321,22 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             }
         } else if (ok && nkb > 0) {
             const int quad = warp & 3;
-
-            const int f = tile * kBlockM + quad * 32 + lane;
-            const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
-            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld16(lane_addr + (uint32_t)c0, v);
-                if (f < p.n_out) {
+            for (int a = 0; a < p.mt; ++a) {
+                const int f = (tile * p.mt + a) * kBlockM + quad * 32 + lane;
+                const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * p.acc_cols);
+                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_addr + (uint32_t)c0, v);
+                    if (f < p.n_out) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const int j = c0 + c;
-                        if (j < p.m) {
-                            const float val = __uint_as_float(v[c]);
-                            if (EPI == kEpiStore) p.Y[(size_t)j * p.ldy + f] = val;
-                            else if (EPI == kEpiAtomic) atomicAdd(p.Y + (size_t)j * p.ldy + f, val);
-                            else atomicAdd(p.Y + (size_t)p.idx[j] * p.ldy + f, val);
+                        for (int c = 0; c < 16; ++c) {
+                            const int j = c0 + c;
+                            if (j < p.m) {
+                                const float val = __uint_as_float(v[c]);
+                                if (EPI == kEpiStore) p.Y[(size_t)j * p.ldy + f] = val;
+                                else if (EPI == kEpiAtomic) atomicAdd(p.Y + (size_t)j * p.ldy + f, val);
+                                else atomicAdd(p.Y + (size_t)p.idx[j] * p.ldy + f, val);
+                            }
                         }
                     }
                 }

@@ -164,6 +164,16 @@ def test_decode_bf16_gqa_ragged(shape):
     assert agrees.mean() >= 0.9  # tiny vocab-independent sanity; the aggregate bar is checked at scale
 
 
+@pytest.mark.parametrize("B", [70, 200])
+def test_decode_bf16_many_rows_two_tile_projection(B):
+    """Enough active rows that a projection CTA takes two weight tiles per activation tile."""
+    shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
+    lens = fi.prompt_lengths(B, 1, 90, 13)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.85, 14)
+    errs, agrees = _run_decode_case(shape, True, lens, mask, 2, 16, 2e-2)
+    assert agrees.mean() >= 0.98
+
+
 def test_all_skip_and_all_keep_masks():
     shape = fi.TINY
     lens = [5, 9]
