@@ -35,6 +35,9 @@ WORKLOADS = {
     "cfg1_1b_b1": dict(shape="1b", B=1, lo=512, hi=512, steps=256, mask=("fraction", 0.25, 0.25)),
     "cfg2_8b_b32": dict(shape="8b", B=32, lo=128, hi=2048, steps=128, mask=("fraction", 0.10, 0.40)),
     "cfg3_8b_b256": dict(shape="8b", B=256, lo=1024, hi=4096, steps=64, mask=("bernoulli", 0.7)),
+    # small-cache cases for profiler captures of the projections at a given row count (not benchmark lines)
+    "prof_8b_b192": dict(shape="8b", B=192, lo=64, hi=128, steps=8, mask=("dense",)),
+    "prof_8b_b64": dict(shape="8b", B=64, lo=64, hi=128, steps=8, mask=("dense",)),
     "cfg4_8b_b64": dict(shape="8b", B=64, lo=1024, hi=1024, steps=128, mask=("aligned", 0.25)),
 }
 SHAPES = {"1b": fi.LLAMA_1B, "8b": fi.LLAMA_8B, "3b": fi.LLAMA_3B}
