@@ -243,6 +243,13 @@ const char *first_kernel_class_name(int32_t k);
  *                    (tokens, outputs, cache tensors) and plan, as a CUDA graph, and
  *                    replays it; up to 8 such graphs are kept.  Nothing is captured while the
  *                    caller's stream is itself being captured or while first_profile is on.
+ *   "tc_lo_max_rows" the hi/lo activation split is used for projections with at most this many
+ *                    active rows, the hi half alone above (default: always both halves; the hi
+ *                    half alone is bfloat16-activation accuracy and misses the parity bar)
+ *   "tc_mt2_min_rows" from this many active rows on a projection CTA takes two weight tiles per
+ *                    activation tile (default: never)
+ *   "tc_ksplit_cap"  0 = do not bound the number of K ranges by the reduction traffic
+ *   "tc_smem_kb"     shared-memory budget per projection CTA when two CTAs per SM are wanted (110)
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
  *                    its epilogue (needs ffn_dim % 64 == 0).

@@ -92,7 +92,9 @@ struct first_ctx {
     int tc_use_lo = 1;
     int fuse_swiglu = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
-    int tc_mt2_min_rows = 49;  // from this many active rows on, a projection CTA takes two weight tiles
+    int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
+    int tc_mt2_min_rows = 1 << 30;
+    int tc_ksplit_cap = 1;  // from this many active rows on, a projection CTA takes two weight tiles
 };
 
 constexpr int kSimpleSplitsMax = 16;
@@ -198,12 +200,18 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
 
 constexpr int kTcSmemMax = 210 * 1024;
 
+// K ranges per weight tile for the reducing epilogues.  More ranges fill the SMs when a matrix has
+// few tiles, but every range adds m*n_out float32 reductions: keep that traffic below about half
+// of the weight bytes (ksplit <= K / (4 m)).
 int tc_ksplit(const first_ctx* c, int n_out, int K, int epi, int m) {
-    if (epi == tc::kEpiStore) return 1;
-    const int mt = (std::min(m, 256) >= c->tc_mt2_min_rows) ? 2 : 1;
+    if (epi == tc::kEpiStore || epi == tc::kEpiSwiglu) return 1;
+    m = std::min(m, 256);
+    const int mt = (m >= c->tc_mt2_min_rows) ? 2 : 1;
     const int tiles = (n_out + tc::kBlockM * mt - 1) / (tc::kBlockM * mt), kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
-    const int ks = (2 * c->n_sm + tiles / 2) / tiles;
-    return std::max(1, std::min(ks, kblocks / 4));
+    int ks = (2 * c->n_sm + tiles / 2) / tiles;
+    ks = std::min(ks, kblocks / 4);
+    if (c->tc_ksplit_cap) ks = std::min(ks, std::max(1, K / (4 * std::max(m, 1))));
+    return std::max(1, ks);
 }
 
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
@@ -220,16 +228,12 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.n_out = n_out; p.K = K; p.m = mm;
         p.n_pad = (mm + 15) / 16 * 16;
         p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
-        p.use_lo = c->tc_use_lo ? 1 : 0;
+        p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
         p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
         if (epi == tc::kEpiSwiglu && n_out % 128) p.mt = 1;
         const int tile_rows = (epi == tc::kEpiSwiglu ? 64 : tc::kBlockM) * p.mt;
         const int tiles = (n_out + tile_rows - 1) / tile_rows;
-        p.ksplit = 1;
-        if (epi != tc::kEpiSwiglu && epi != tc::kEpiStore) {
-            const int ks = (2 * c->n_sm + tiles / 2) / tiles;
-            p.ksplit = std::max(1, std::min(ks, p.kblocks / 4));
-        }
+        p.ksplit = tc_ksplit(c, n_out, K, epi, mm);
         p.act = act ? act + (size_t)r0 * n_out : nullptr;
         p.act_hi = act_hi ? act_hi + (size_t)r0 * n_out : nullptr;
         p.act_lo = act_lo ? act_lo + (size_t)r0 * n_out : nullptr;
@@ -794,7 +798,9 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
     else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
-    else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : 49;
+    else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
+    else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : (1 << 30);
+    else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
     else return FIRST_E_ARG;
     c->plan_version += 1;  // cached step graphs were built under the old options
