@@ -372,7 +372,18 @@ def run_cuda(args, wl, shape, mask, lens):
     if cls_ms.get("gemv_rows") and cls_ms.get("gemm_tc"):
         alg = {"attn_split": bm["kv"]}  # projections split over two classes: attribute by class below
     dom = max(cls_ms, key=cls_ms.get)
-    roof = {"bound": "hbm", "kernel": dom, "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "traffic": None,
+    traffic = None
+    try:  # DRAM bytes of the projection launches from the committed ncu capture, if the kernel is unchanged since
+        import hashlib
+        tj = json.loads((ROOT / "profiles" / "traffic_gemm_tc_cfg2.json").read_text())
+        cur = hashlib.sha256((ROOT / tj["source"]).read_bytes()).hexdigest()[:16]
+        if dom == "gemm_tc" and cur == tj["source_sha256_16"] and wl["shape"] == "8b":
+            bl = tj["bytes_per_launch"]
+            traffic = int((cnt > 0).sum()) * (bl["qkv"] + bl["o"] + bl["gate_up"] + bl["down"]) + bl["lm_head"]
+    except Exception:
+        traffic = None
+    roof = {"bound": "hbm", "kernel": dom, "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "traffic": traffic,
+            "traffic_note": "per step, scaled from the 2-layer ncu capture in profiles/ (per launch x launches)" if traffic else None,
             "ms_per_step": cls_ms[dom], "share_of_kernel_time": cls_ms[dom] / tot_cls}
     if dom in alg:
         roof["achieved"] = alg[dom] / cls_ms[dom] / 1e6
