@@ -660,6 +660,9 @@ int first_set_mask(first_ctx* c, const uint8_t* mask, int32_t B, void* stream) {
     if (B > c->d.max_batch) return FIRST_E_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c->has_mask = false;
+    c->plan_version += 1;  // step graphs recorded under the previous plan must not be replayed
+    for (auto& e : c->graphs) cudaGraphExecDestroy(e.exec);
+    c->graphs.clear();
     FIRST_LAUNCH(kClsPlan, (plan_compact<<<c->d.n_layers, 32, 0, st>>>(mask, B, c->d.n_layers, c->idx, c->cnt, c->slot, c->flags)));
     int rc = check_launch(c);
     if (rc) return rc;

@@ -210,6 +210,31 @@ def test_batch_rows_are_independent_on_gpu():
     assert np.array_equal(run([1])[0], base[1])
 
 
+def test_new_mask_with_the_same_buffers_takes_effect():
+    """A second first_set_mask on the same context, with the same token / cache / logits buffers,
+    must change what the next step computes (cached launch sequences belong to the old plan)."""
+    import torch
+    shape = fi.TINY
+    w = fi.make_weights(shape, 2, False)
+    om = oracle_model(shape, w)
+    lens = [6, 11, 3]
+    ctx = _ctx(shape, False, 3, 32, w)
+    toks = np.array([3, 4, 5], np.int32)
+    t_dev = torch.from_numpy(toks).cuda()
+    logits = torch.empty((3, shape.vocab), dtype=torch.float32, device="cuda")
+    masks = [np.ones((3, shape.n_layers), np.uint8), np.array([[1, 0, 0, 1], [0, 0, 1, 1], [1, 1, 0, 0]], np.uint8),
+             np.zeros((3, shape.n_layers), np.uint8)]
+    okv, gkv = synthetic_caches(shape, lens, [n + 8 for n in lens], 3, False)
+    for mk in masks:
+        ctx.set_mask(torch.from_numpy(mk).cuda())
+        for _ in range(2):  # twice: the second call replays what the first recorded
+            ref = oracle.decode_step(om, toks, mk, okv)
+            ctx.decode_step(t_dev, gkv.c, logits)
+            err, agree = logits_check(logits.cpu().numpy(), ref)
+            assert err.max() <= 1e-4 and agree.all()
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
+
+
 def test_full_slab_sets_flag_and_leaves_cache():
     import torch
     shape = fi.TINY
