@@ -312,6 +312,18 @@ def run_cuda(args, wl, shape, mask, lens):
     repeat_ms, _ = timed(mask_t)  # the routed run once more, after the dense one (order effects show here)
     repeat_ms /= K
 
+    sweep = None
+    if args.sweep:
+        sweep = []
+        for frac in (0.0, 0.1, 0.2, 0.3, 0.4, 0.5):
+            row = {"skip": frac}
+            for kind in ("aligned", "independent"):
+                mk = fi.mask_aligned(B, L, frac) if kind == "aligned" else fi.mask_independent(B, L, frac, 3000 + rank)
+                ms, _ = timed(torch.from_numpy(mk).to(dev))
+                bmk = byte_model(shape, mk, lens + W + K // 2)
+                row[kind] = {"ms_per_step": ms / K, "bytes_strict": bmk["strict"]}
+            sweep.append(row)
+
     # ---- end to end through the public call with host buffers
     ctx.set_mask(mask_t)
     reset()
@@ -414,7 +426,7 @@ def run_cuda(args, wl, shape, mask, lens):
            "dense": {"ms_per_step": dense_ms, "gpu_launches": int(dense_launches), "bytes_strict": bm_dense["strict"],
                      "latency_ratio_routed_over_dense": ms_step / dense_ms,
                      "bytes_ratio_routed_over_dense": bm["full"] / bm_dense["full"]},
-           "ms_per_step_repeat": repeat_ms,
+           "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
            "kernel_ms_per_step": cls_ms, "route": route}
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5)
@@ -437,6 +449,8 @@ def main():
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (A/B runs)")
     ap.add_argument("--layers", type=int, default=None,
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also time skip fractions 0..50 %% (aligned and independent masks) on this workload")
     ap.add_argument("--quick", action="store_true",
                     help="only the main timed loop (for profiler captures): no dense/e2e/per-kernel legs")
     args = ap.parse_args()
