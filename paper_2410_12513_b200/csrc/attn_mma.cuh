@@ -104,6 +104,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     if (warp == 4) {  // ---------------- producer
         if (lane == 0) {
             const int64_t row0 = (int64_t)h * cap_total + slab_off[b] + t_begin;
+            uint64_t pol;  // cached keys/values are read once per step: do not let them displace L2 contents
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
             int issued = 0;
             for (int j = 0; j < n_tiles; ++j, ++issued) {
                 const int s = j % kStages;
@@ -114,8 +116,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                 const int row = (int)(row0 + (int64_t)j * kTile);
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tc::tma_load_2d(sa + hf * kBox, &tmK, full_bar(s), hf * 64, row);
-                    tc::tma_load_2d(sa + (kHalves + hf) * kBox, &tmV, full_bar(s), hf * 64, row);
+                    tc::tma_load_2d_hint(sa + hf * kBox, &tmK, full_bar(s), hf * 64, row, pol);
+                    tc::tma_load_2d_hint(sa + (kHalves + hf) * kBox, &tmV, full_bar(s), hf * 64, row, pol);
                 }
             }
             if (abort_s) {
