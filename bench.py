@@ -73,6 +73,21 @@ def byte_model(shape, mask, lens, kv_elem=2, w_elem=2):
     return dict(strict=strict, full=full, weights=weights, kv=kv, lm_head=shape.vocab * shape.d_model * w_elem)
 
 
+def max_over_ranks(ms, dist, device):
+    """Slowest rank's time (replicas run independently; the job is as slow as its slowest GPU)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(world, batch_per_rank, steps, ms_max):
+    """Whole-job throughput of `world` replicas, each decoding `batch_per_rank` sequences for `steps` steps."""
+    return world * batch_per_rank * steps / (ms_max / 1e3)
+
+
 class ClockSampler:
     """nvidia-smi sampled every 200 ms while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -266,10 +281,7 @@ def run_cuda(args, wl, shape, mask, lens):
         barrier()
         ms = e0.elapsed_time(e1)
         launches = ctx.launch_count() - l0
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ms, dist, dev)
         return ms, launches
 
     # ---- routing + plan, once per batch (reported, not part of the step)
@@ -300,7 +312,7 @@ def run_cuda(args, wl, shape, mask, lens):
         ms_total, launches = timed(mask_t)
     clocks = sampler.summary()
     ms_step = ms_total / K
-    value = world * B * K / (ms_total / 1e3)
+    value = job_tokens_per_s(world, B, K, ms_total)
 
     if args.quick:
         if rank == 0:
@@ -346,11 +358,8 @@ def run_cuda(args, wl, shape, mask, lens):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * B * K / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": B * 4,
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    e2e = {"value": job_tokens_per_s(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": B * 4,
            "d2h_bytes_per_step": B * 4, "ms_per_step": e2e_ms / K}
 
     # ---- per-kernel-class device time (separate pass: event pairs around every launch)
