@@ -49,7 +49,7 @@ __device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, 128;
 
 // grid (S_max, Hkv, m), 160 threads.  Work item = (active row i, kv head h, chunk c):
 // tokens [c*C, min(T, (c+1)*C)), T = len[b]+1 (the new token was just written at row len[b];
-// T = len[b] if the slab was full and nothing was written).  Chunks past T exit at once.
+// T = len[b] if the slab was full and nothing was written), taken from rowinfo[i].  Chunks past T exit at once.
 // q: [m][Hq][HD] float32, pre-scaled by 1/sqrt(HD).  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64x64.
 // Scratch: o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum),
 // ticket [m][Hkv] (zero between launches: the merging CTA resets it).
@@ -58,10 +58,7 @@ template <int HD, int G>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
                                                       const float* __restrict__ q, int64_t cap_total,
-                                                      const int64_t* __restrict__ slab_off,
-                                                      const int32_t* __restrict__ len_l,
-                                                      const int32_t* __restrict__ slab_cap,
-                                                      const int32_t* __restrict__ idx, int Hq, int C,
+                                                      const longlong2* __restrict__ rowinfo, int Hq, int C,
                                                       float* __restrict__ o_part, float2* __restrict__ ml_part,
                                                       uint32_t* __restrict__ ticket, float* __restrict__ out,
                                                       __nv_bfloat16* __restrict__ out_hi,
@@ -76,8 +73,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     pdl_trigger();
     pdl_wait();
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
-    const int b = idx[i];
-    const int T = min(len_l[b] + 1, slab_cap[b]);
+    const longlong2 ri = rowinfo[i];  // (tokens present incl. the new one, first slab row), written by rope_append
+    const int T = (int)ri.x;
     const int t_begin = c * C;
     if (t_begin >= T) return;
     const int n_chunks = (T + C - 1) / C;
@@ -103,7 +100,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
 
     if (warp == 4) {  // ---------------- producer
         if (lane == 0) {
-            const int64_t row0 = (int64_t)h * cap_total + slab_off[b] + t_begin;
+            const int64_t row0 = (int64_t)h * cap_total + ri.y + t_begin;
             uint64_t pol;  // cached keys/values are read once per step: do not let them displace L2 contents
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
             int issued = 0;

@@ -59,6 +59,7 @@ struct first_ctx {
     double* inv_freq = nullptr;
     int32_t *idx = nullptr, *cnt = nullptr, *slot = nullptr;
     uint32_t *flags = nullptr, *ticket = nullptr;
+    longlong2* rowinfo = nullptr;  // per active row: (tokens to attend over, first slab row)
     int64_t tok_cap = 0;
     int max_splits = 16;
     int attn_chunk = -1;
@@ -358,7 +359,7 @@ int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorM
                        __nv_bfloat16* out_hi, __nv_bfloat16* out_lo) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
-                    kv->slab_off, len_l, kv->slab_cap, idx, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
+                    c->rowinfo, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
                     out_hi, out_lo, c->flags);
 }
 
@@ -441,6 +442,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     int S = (d.max_tokens_per_seq + 255) / 256;
     S = std::max(1, std::min(S, kSimpleSplitsMax));
     const float qscale = 1.0f / std::sqrt((float)hd);
+    const int norm_threads = std::max(32, std::min(1024, (D / 4 + 31) / 32 * 32));  // one float4 per thread when the row allows
     const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
 
     for (int l = 0; l < L; ++l) {
@@ -461,7 +463,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
         const bool zero_gu = t && !fused_ffn && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic, m) > 1;
         // ---- attention half
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->attn_norm[l],
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
@@ -470,7 +472,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         if ((rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
                            0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total, kv->slab_off,
-                           kv->slab_cap, len_l, c->flags)))
+                           kv->slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr)))
             return rc;
         if (mma_attn) {
             if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, t ? nullptr : c->att, xh, xl)))
@@ -485,7 +487,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                               D, idx)))
             return rc;
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(256), 0, c->x, idx, D, c->ffn_norm[l],
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->ffn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap)))
             return rc;
         if (fused_ffn) {
@@ -509,7 +511,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     float* lg = logits ? logits : (next_tokens ? c->logits_int : nullptr);
     if (lg) {
         const bool t = tc_for(B);
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(256), 0, c->x, nullptr, D, c->final_norm,
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, D, c->final_norm,
                            d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
                            nullptr)))
             return rc;
@@ -593,7 +595,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         (rc = dev_alloc(&c->cs, MB * (d.head_dim / 2))) || (rc = dev_alloc(&c->inv_freq, (size_t)d.head_dim / 2)) ||
         (rc = dev_alloc(&c->idx, MB * d.n_layers)) || (rc = dev_alloc(&c->cnt, (size_t)d.n_layers)) ||
         (rc = dev_alloc(&c->slot, MB * d.n_layers)) || (rc = dev_alloc(&c->flags, (size_t)1)) ||
-        (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)))
+        (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)) || (rc = dev_alloc(&c->rowinfo, MB)))
         return fail(rc);
     if (cudaMemset(c->ticket, 0, MB * d.n_kv_heads * sizeof(uint32_t)) != cudaSuccess) return fail(FIRST_E_CUDA);
     if (d.dtype == FIRST_DTYPE_BF16) {
@@ -617,7 +619,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
 int first_destroy(first_ctx* c) {
     if (!c) return FIRST_OK;
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
-                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket};
+                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket, c->rowinfo};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);

@@ -57,44 +57,66 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 //   zero_row: row i of a float32 accumulator (zero_cols wide) is cleared for a split-K projection;
 //   len_inc:  the row's cache length is advanced by one (unless its slab is full) -- done here,
 //             after the layer's attention, so no attention block can see a half-updated length.
-__global__ void __launch_bounds__(256) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
-                                                    const float* __restrict__ gain, float eps, float* __restrict__ out,
-                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
-                                                    float* __restrict__ zero_row, int zero_cols,
-                                                    int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap) {
+__global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
+                                                     const float* __restrict__ gain, float eps, float* __restrict__ out,
+                                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                     float* __restrict__ zero_row, int zero_cols,
+                                                     int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap) {
+    // One pass: the row stays in registers between the sum of squares and the scaling
+    // (up to kMaxV float4 per thread; longer rows re-read the tail from L1/L2).
+    constexpr int kMaxV = 4;
     pdl_trigger();
+    const int i = blockIdx.x, nt = blockDim.x;
+    float4 g[kMaxV];
+    const int nv = D / 4;
+#pragma unroll
+    for (int v = 0; v < kMaxV; ++v) {  // gains do not depend on the previous kernel: fetch them before the wait
+        const int k = threadIdx.x + v * nt;
+        if (k < nv) g[v] = __ldg(reinterpret_cast<const float4*>(gain) + k);
+    }
     pdl_wait();
-    __shared__ float red[8];
-    const int i = blockIdx.x;
+    __shared__ float red[32];
     const int b = idx ? idx[i] : i;
     if (len_inc && threadIdx.x == 0) {
         const int T = len_inc[b];
         if (T < slab_cap[b]) len_inc[b] = T + 1;
     }
-    if (zero_row) {
-        float4* z = reinterpret_cast<float4*>(zero_row + (size_t)i * zero_cols);
-        for (int k = threadIdx.x; k < zero_cols / 4; k += 256) z[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    const float* xr = x + (size_t)b * D;
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)b * D);
+    float4 r[kMaxV];
     float ss = 0.f;
-    for (int k = threadIdx.x * 4; k < D; k += 1024) {
-        const float4 v = *reinterpret_cast<const float4*>(xr + k);
+#pragma unroll
+    for (int v = 0; v < kMaxV; ++v) {
+        const int k = threadIdx.x + v * nt;
+        if (k < nv) {
+            r[v] = xr[k];
+            ss += r[v].x * r[v].x + r[v].y * r[v].y + r[v].z * r[v].z + r[v].w * r[v].w;
+        }
+    }
+    for (int k = threadIdx.x + kMaxV * nt; k < nv; k += nt) {
+        const float4 v = xr[k];
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    if (zero_row) {
+        float4* z = reinterpret_cast<float4*>(zero_row + (size_t)i * zero_cols);
+        for (int k = threadIdx.x; k < zero_cols / 4; k += nt) z[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     __syncthreads();
     float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
+    for (int w = 0; w < (nt >> 5); ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)D + eps);
-    for (int k = threadIdx.x * 4; k < D; k += 1024) {
-        const float4 v = *reinterpret_cast<const float4*>(xr + k);
-        const float4 g = *reinterpret_cast<const float4*>(gain + k);
-        const float y[4] = {v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w};
-        if (out) *reinterpret_cast<float4*>(out + (size_t)i * D + k) = make_float4(y[0], y[1], y[2], y[3]);
-        if (hi) split_store4(y, hi + (size_t)i * D + k, lo + (size_t)i * D + k);
+    auto emit = [&](int k, const float4& v, const float4& gg) {
+        const float y[4] = {v.x * inv * gg.x, v.y * inv * gg.y, v.z * inv * gg.z, v.w * inv * gg.w};
+        if (out) *reinterpret_cast<float4*>(out + (size_t)i * D + 4 * k) = make_float4(y[0], y[1], y[2], y[3]);
+        if (hi) split_store4(y, hi + (size_t)i * D + 4 * k, lo + (size_t)i * D + 4 * k);
+    };
+#pragma unroll
+    for (int v = 0; v < kMaxV; ++v) {
+        const int k = threadIdx.x + v * nt;
+        if (k < nv) emit(k, r[v], g[v]);
     }
+    for (int k = threadIdx.x + kMaxV * nt; k < nv; k += nt) emit(k, xr[k], __ldg(reinterpret_cast<const float4*>(gain) + k));
 }
 
 // After the QKV projection: rotate q and k at the sequence's position, scale q by
@@ -102,6 +124,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows(const float* __restrict__ x,
 // qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  grid (Hq+2*Hkv, m): one block of
 // hd/2 threads per (row, head); thread d handles the rotary pair (d, d+hd/2).
 // len is only read here (the FFN-side rmsnorm_rows advances it once attention is done).
+// rowinfo[i] = (tokens to attend over, first slab row) saves the attention CTAs two dependent loads.
 // A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
 __global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv, const int32_t* __restrict__ idx,
@@ -110,10 +133,13 @@ __global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv,
                                                   KT* __restrict__ vc, int64_t cap_total,
                                                   const int64_t* __restrict__ slab_off,
                                                   const int32_t* __restrict__ slab_cap,
-                                                  const int32_t* __restrict__ len_l, uint32_t* __restrict__ flags) {
+                                                  const int32_t* __restrict__ len_l, uint32_t* __restrict__ flags,
+                                                  longlong2* __restrict__ rowinfo) {
     pdl_trigger();
     pdl_wait();
     const int i = blockIdx.y, head = blockIdx.x, d = threadIdx.x, b = idx[i];
+    if (rowinfo && head == 0 && d == 0)  // what attention needs to know about this row, in one 16-byte word
+        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]), (long long)slab_off[b]);
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
     const float* row = qkv + (size_t)i * (qd + 2 * kvd) + (size_t)head * hd;
