@@ -53,6 +53,7 @@ struct first_ctx {
     std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wgu64, tm_wd;  // tm_wgu64: 64-row boxes (gate|up pairing)
     CUtensorMap tm_lm{};
     bool tc_ready = false;
+    int pair_rows = 64;  // gate (= up) rows per tile of the fused gate/up projection; tm_wgu64 has boxes of this many rows
     struct KvMap { int64_t cap_total; CUtensorMap map; };
     std::unordered_map<const void*, KvMap> kv_maps;  // TMA descriptors of cache tensors, by base pointer
     float2 *ml_part = nullptr, *cs = nullptr;
@@ -92,6 +93,7 @@ struct first_ctx {
     int attn_simple = -1;
     int tc_use_lo = 1;
     int fuse_swiglu = 1;
+    int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
     int tc_mt2_min_rows = 1 << 30;
@@ -232,7 +234,8 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
         p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
         if (epi == tc::kEpiSwiglu && n_out % 128) p.mt = 1;
-        const int tile_rows = (epi == tc::kEpiSwiglu ? 64 : tc::kBlockM) * p.mt;
+        p.pair_rows = c->pair_rows;
+        const int tile_rows = epi == tc::kEpiSwiglu ? (p.mt == 1 ? c->pair_rows : 128) : tc::kBlockM * p.mt;
         const int tiles = (n_out + tile_rows - 1) / tile_rows;
         p.ksplit = tc_ksplit(c, n_out, K, epi, mm);
         p.act = act ? act + (size_t)r0 * n_out : nullptr;
@@ -275,12 +278,19 @@ int tc_setup(first_ctx* c) {
     const first_model_desc& d = c->d;
     int rc;
     const int L = d.n_layers;
+    // Rows per half-tile of the fused gate/up projection: as large as 64, but small enough that the
+    // tiles fill two CTA slots per SM in a single wave (8B shape on 148 SMs: 49 rows -> 293 tiles).
+    c->pair_rows = 64;
+    if (c->tune_pair_rows && d.ffn_dim > 64 * c->n_sm) {
+        const int want = (d.ffn_dim + 2 * c->n_sm - 1) / (2 * c->n_sm);
+        if (want <= 64) c->pair_rows = std::max(8, want);
+    }
     c->tm_wqkv.resize(L); c->tm_wo.resize(L); c->tm_wgu.resize(L); c->tm_wgu64.resize(L); c->tm_wd.resize(L);
     for (int l = 0; l < L; ++l) {
         if ((rc = make_map(&c->tm_wqkv[l], c->wqkv[l], c->qkvd, d.d_model, tc::kBlockM, true)) ||
             (rc = make_map(&c->tm_wo[l], c->wo[l], d.d_model, c->qd, tc::kBlockM, true)) ||
             (rc = make_map(&c->tm_wgu[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, tc::kBlockM, true)) ||
-            (rc = make_map(&c->tm_wgu64[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, 64, true)) ||
+            (rc = make_map(&c->tm_wgu64[l], c->w_gate_up[l], 2 * (uint64_t)d.ffn_dim, d.d_model, c->pair_rows, true)) ||
             (rc = make_map(&c->tm_wd[l], c->w_down[l], d.d_model, d.ffn_dim, tc::kBlockM, true)))
             return rc;
     }

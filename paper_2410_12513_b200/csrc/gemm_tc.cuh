@@ -45,6 +45,8 @@ struct GemmParams {
     uint32_t* flags;
     // kEpiSwiglu: the weight matrix is [gate rows (n_out) | up rows (n_out)]; a tile pairs 64 gate
     // features with the same 64 up features and the epilogue writes silu(gate)*up:
+    int pair_rows;           // gate rows (= up rows) per tile when mt == 1: at most 64, chosen so that the
+                             // tiles fill the GPU's CTA slots in one wave
     float* act;              // [m][n_out] float32 or NULL
     __nv_bfloat16* act_hi;   // [m][n_out] bfloat16 hi/lo split or NULL
     __nv_bfloat16* act_lo;
@@ -170,14 +172,16 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
         if (lane == 0) {
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            const uint32_t tx = (uint32_t)stage_bytes;
+            const uint32_t tx = (EPI == kEpiSwiglu && p.mt == 1)
+                                    ? (uint32_t)(stage_bytes - a_bytes + 2 * p.pair_rows * 128)  // two boxes of R rows
+                                    : (uint32_t)stage_bytes;
             auto load_a = [&](uint32_t sa, uint32_t bar, int kc) {
                 if (EPI == kEpiSwiglu) {
-                    // gate rows, then the matching up rows: 64+64 (mt = 1) or 128+128 (mt = 2)
-                    const int rows = 64 * p.mt;
+                    // gate rows, then the matching up rows: R+R (mt = 1, R = pair_rows <= 64) or 128+128 (mt = 2)
+                    const int rows = p.mt == 1 ? p.pair_rows : 128;
                     const CUtensorMap* tm = p.mt == 1 ? &tmA : &tmA2;
                     tma_load_2d_hint(sa, tm, bar, kc, tile * rows, pol_stream);
-                    tma_load_2d_hint(sa + a_bytes / 2, tm, bar, kc, p.n_out + tile * rows, pol_stream);
+                    tma_load_2d_hint(sa + rows * 128, tm, bar, kc, p.n_out + tile * rows, pol_stream);
                 } else {
                     for (int a = 0; a < p.mt; ++a)
                         tma_load_2d_hint(sa + a * kABytes, &tmA, bar, kc, (tile * p.mt + a) * kBlockM, pol_stream);
@@ -277,36 +281,38 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 }
             }
         } else if (EPI == kEpiSwiglu) {
-            // lanes 0..63 of the accumulator hold gate features, lanes 64..127 the matching up features.
-            // Up warps park their values in shared memory (the ring is idle once the accumulator is
-            // complete), gate warps combine.  u_s[j][feature]: conflict-free both ways.
-            const int quad = warp & 3;
+            // lanes [0, R) of the accumulator hold gate features, lanes [R, 2R) the matching up features
+            // (R = pair_rows; lanes from 2R up saw stale shared memory and are ignored).  Up lanes park
+            // their values in shared memory (the ring is idle once the accumulator is complete), gate
+            // lanes combine.  u_s[j][feature]: conflict-free both ways.
+            const int quad = warp & 3, R = p.pair_rows;
             float* u_s = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)));
             const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
             const bool run = ok && nkb > 0;
-            if (quad >= 2 && run) {
-                const int fl = (quad - 2) * 32 + lane;
+            const int gl = quad * 32 + lane;  // accumulator lane of this thread
+            if (run && quad * 32 + 31 >= R && quad * 32 < 2 * R) {  // this warp holds some up lanes
                 for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld16(lane_addr + (uint32_t)c0, v);
+                    if (gl >= R && gl < 2 * R) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) u_s[(c0 + c) * 64 + fl] = __uint_as_float(v[c]);
+                        for (int c = 0; c < 16; ++c) u_s[(c0 + c) * 64 + (gl - R)] = __uint_as_float(v[c]);
+                    }
                 }
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");
-            if (quad < 2 && run) {
-                const int fl = quad * 32 + lane;
-                const int f = tile * 64 + fl;
+            if (run && quad * 32 < R) {  // this warp holds some gate lanes
+                const int f = tile * R + gl;
                 for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld16(lane_addr + (uint32_t)c0, v);
-                    if (f < p.n_out) {
+                    if (gl < R && f < p.n_out) {
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             const int j = c0 + c;
                             if (j < p.m) {
                                 const float g = __uint_as_float(v[c]);
-                                const float y = g / (1.f + expf(-g)) * u_s[j * 64 + fl];
+                                const float y = g / (1.f + expf(-g)) * u_s[j * 64 + gl];
                                 const size_t o = (size_t)j * p.n_out + f;
                                 if (p.act) p.act[o] = y;
                                 if (p.act_hi) {
