@@ -234,7 +234,9 @@ const char *first_kernel_class_name(int32_t k);
 
 /* Options (A/B measurements and tuning).  A negative value restores the default.
  *   "max_gemv_rows"  largest active-row count served by the CUDA-core GEMV path; layers with
- *                    more rows use the tensor-core path when the dtype is bfloat16 (default 2)
+ *                    more rows use the tensor-core path when the dtype is bfloat16 (default 0: with TMA streaming
+ *                    and weight prefetch across kernel boundaries it is the faster path even for one row;
+ *                    float32 models always use the GEMV path)
  *   "attn_simple"    1 = always use the general attention kernel
  *   "attn_chunk"     tokens per attention work item (rounded up to 64); default: from the batch
  *   "tc_use_lo"      0 = tensor-core projections use only the bfloat16 hi half of activations

@@ -401,6 +401,8 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
         const double est = 0.6 * (double)m * d.n_kv_heads * d.max_tokens_per_seq;
         C = (int)(est / (4.0 * c->n_sm));
         C = std::max(512, std::min(2048, C));
+        // few rows: smaller chunks until there is at least one work item per SM
+        while (C > 128 && est / C < c->n_sm) C /= 2;
     }
     C = std::max(C, (d.max_tokens_per_seq + c->max_splits - 1) / c->max_splits);
     C = (C + attn::kTile - 1) / attn::kTile * attn::kTile;
@@ -441,7 +443,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const first_model_desc& d = c->d;
     const int B = c->B, D = d.d_model, F = d.ffn_dim, V = d.vocab, L = d.n_layers, hd = d.head_dim;
     constexpr bool kBf16 = std::is_same<WT, __nv_bfloat16>::value;
-    const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 2;
+    const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 0;
     auto tc_for = [&](int m) { return kBf16 && c->tc_ready && m > gemv_max; };
     int rc;
     c->pdl_next = false;  // the first kernel of a step has no predecessor to overlap

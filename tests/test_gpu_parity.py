@@ -174,6 +174,15 @@ def test_decode_bf16_many_rows_two_tile_projection(B):
     assert agrees.mean() >= 0.98
 
 
+def test_decode_bf16_gemv_path_and_general_attention_by_option():
+    """The CUDA-core GEMV projections and the general attention kernel, forced by option, on a bf16 model."""
+    shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
+    lens = fi.prompt_lengths(5, 1, 200, 23)
+    mask = fi.mask_bernoulli(5, shape.n_layers, 0.7, 24)
+    _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"max_gemv_rows": 8, "attn_simple": 1})
+    _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"fuse_swiglu": 0, "use_pdl": 0, "use_graph": 0})
+
+
 def test_all_skip_and_all_keep_masks():
     shape = fi.TINY
     lens = [5, 9]
