@@ -38,6 +38,8 @@ WORKLOADS = {
     # small-cache cases for profiler captures of the projections at a given row count (not benchmark lines)
     "prof_8b_b192": dict(shape="8b", B=192, lo=64, hi=128, steps=8, mask=("dense",)),
     "prof_8b_b64": dict(shape="8b", B=64, lo=64, hi=128, steps=8, mask=("dense",)),
+    # the paper's second model shape (Llama-3.2-3B: 28 layers, 24 query / 8 KV heads), config-2-like batch
+    "llama3b_b32": dict(shape="3b", B=32, lo=128, hi=2048, steps=128, mask=("fraction", 0.10, 0.40)),
     "cfg4_8b_b64": dict(shape="8b", B=64, lo=1024, hi=1024, steps=128, mask=("aligned", 0.25)),
 }
 SHAPES = {"1b": fi.LLAMA_1B, "8b": fi.LLAMA_8B, "3b": fi.LLAMA_3B}
@@ -53,6 +55,10 @@ def make_mask(recipe, B, L, seed):
         return fi.mask_aligned(B, L, recipe[1])
     if kind == "independent":
         return fi.mask_independent(B, L, recipe[1], seed)
+    if kind == "unified":
+        return fi.mask_unified(B, L, int(recipe[1]))
+    if kind == "random":
+        return fi.mask_random_shared(B, L, recipe[1], 2000)  # one draw for the whole job, every rank the same
     if kind == "dense":
         return np.ones((B, L), np.uint8)
     raise ValueError(kind)
@@ -452,7 +458,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2_8b_b32", choices=sorted(WORKLOADS))
-    ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI")
+    ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI | bernoulli:P | unified:EVERY | random:F")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-route", action="store_true")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (A/B runs)")

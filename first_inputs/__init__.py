@@ -188,6 +188,29 @@ def mask_independent(B: int, L: int, frac: float, seed: int) -> np.ndarray:
     return mask_skip_fraction(B, L, frac, frac, seed)
 
 
+def mask_unified(B: int, L: int, every: int) -> np.ndarray:
+    """Input-agnostic preset: every sequence skips the same evenly spaced layers, every
+    `every`-th one counted from layer 1 (first and last layer kept). The fixed-interval
+    skipping strategy the paper compares against (Section 4, baselines)."""
+    m = np.ones((B, L), dtype=np.uint8)
+    if every > 0:
+        for l in range(1, L - 1):
+            if l % every == every - 1:
+                m[:, l] = 0
+    return m
+
+
+def mask_random_shared(B: int, L: int, frac: float, seed: int) -> np.ndarray:
+    """Input-agnostic preset: one random set of round(frac*L) layers from 1..L-2, the same
+    for every sequence. The random skipping strategy the paper compares against."""
+    g = _rng(seed, "mask_random_shared")
+    k = min(int(round(frac * L)), max(L - 2, 0))
+    m = np.ones((B, L), dtype=np.uint8)
+    if k:
+        m[:, g.choice(np.arange(1, L - 1), size=k, replace=False)] = 0
+    return m
+
+
 def synthetic_kv_rows(n_tokens: int, kv_dim: int, seed: int, stream: str, bf16: bool = True) -> np.ndarray:
     """Stand-in cache contents N(0,1) for one (layer, sequence, K-or-V): [n_tokens][kv_dim]."""
     return normal((n_tokens, kv_dim), 1.0, seed, stream, bf16)

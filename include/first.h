@@ -113,7 +113,7 @@ typedef struct {
 /* Create a context for one model on the current device: validates the description,
  * borrows the weights, allocates scratch sized by max_batch / max_tokens_per_seq.
  * Errors: FIRST_E_ARG, FIRST_E_SHAPE (head_dim*heads, divisibility), FIRST_E_UNSUPPORTED
- * (head_dim not in {32,64,128}; Hq/Hkv not in {1,2,4,8}; d_model, ffn_dim not multiples
+ * (head_dim not in {32,64,128}; Hq/Hkv not in {1,2,3,4,8}; d_model, ffn_dim not multiples
  * of 8), FIRST_E_CUDA. */
 int first_create(const first_model_desc *desc, const first_weights *weights, first_ctx **out);
 int first_destroy(first_ctx *ctx);

@@ -330,6 +330,7 @@ int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* 
     switch (c->group) {
         FIRST_ATTN_CASE(1)
         FIRST_ATTN_CASE(2)
+        FIRST_ATTN_CASE(3)
         FIRST_ATTN_CASE(4)
         FIRST_ATTN_CASE(8)
         default: return FIRST_E_UNSUPPORTED;
@@ -384,8 +385,8 @@ int attn_mma_set_attr() {
 int attn_mma_setup(first_ctx* c) {
 #define FIRST_ATTN_MMA(HD, G) \
     if (c->d.head_dim == HD && c->group == G) return attn_mma_set_attr<HD, G>();
-    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
-    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
+    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 3) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
+    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 3) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
     return FIRST_OK;
 }
@@ -414,8 +415,8 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
 #define FIRST_ATTN_MMA(HD, G)                 \
     if (d.head_dim == HD && c->group == G)    \
         return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, len_l, idx, C, out, out_hi, out_lo);
-    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
-    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
+    FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 3) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
+    FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 3) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
     return FIRST_E_UNSUPPORTED;
 }
@@ -564,7 +565,7 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
     if (d.n_q_heads % d.n_kv_heads) return FIRST_E_SHAPE;
     const int group = d.n_q_heads / d.n_kv_heads;
     if (d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128) return FIRST_E_UNSUPPORTED;
-    if (group != 1 && group != 2 && group != 4 && group != 8) return FIRST_E_UNSUPPORTED;
+    if (group != 1 && group != 2 && group != 3 && group != 4 && group != 8) return FIRST_E_UNSUPPORTED;
     if (d.d_model % 8 || d.ffn_dim % 8) return FIRST_E_UNSUPPORTED;
     if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->ffn_norm ||
         !w->w_gate_up || !w->w_down)

@@ -37,6 +37,12 @@ def test_mask_recipes_have_the_stated_structure():
     assert (a == a[0]).all() and (32 - a[0].sum()) == 8 and a[0, 0] and a[0, -1]
     i = fi.mask_independent(8, 32, 0.25, 3)
     assert ((32 - i.sum(1)) == 8).all() and not (i == i[0]).all()
+    u = fi.mask_unified(4, 32, 4)     # layers 3, 7, ..., 27 (31 is the last layer and stays)
+    assert (u == u[0]).all() and [l for l in range(32) if not u[0, l]] == list(range(3, 31, 4))
+    assert fi.mask_unified(2, 32, 0).all()
+    r = fi.mask_random_shared(8, 32, 0.25, 5)
+    assert (r == r[0]).all() and (32 - r[0].sum()) == 8 and r[0, 0] and r[0, -1]
+    assert not (r[0] == fi.mask_random_shared(8, 32, 0.25, 6)[0]).all()
     b = fi.mask_bernoulli(256, 32, 0.7, 2)
     assert b[:, 0].all() and b[:, -1].all() and 0.6 < b[:, 1:-1].mean() < 0.8
 

@@ -155,7 +155,9 @@ def test_decode_f32_tiny_ragged(B):
     assert agrees.all()
 
 
-@pytest.mark.parametrize("shape", [fi.TINY_GQA, fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)])
+@pytest.mark.parametrize("shape", [fi.TINY_GQA, fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0),
+                                   fi.ModelShape(2, 384, 6, 2, 64, 512, 1000, 500000.0),    # 3 query heads per KV head
+                                   fi.ModelShape(2, 384, 3, 1, 128, 512, 1000, 500000.0)])  # (the Llama-3.2-3B grouping)
 def test_decode_bf16_gqa_ragged(shape):
     B = 7
     lens = fi.prompt_lengths(B, 1, 300, 3)
@@ -317,3 +319,72 @@ def test_config0_prefill_route_decode_end_to_end():
         toks = oracle.argmax(ref)
     assert ctx.device_flags() == 0
     assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
+
+
+def test_batch_changes_between_steps():
+    """Continuous batching at the step boundary: with one context, a finished sequence's slot is
+    handed to a new sequence with its own mask row, then the batch shrinks by one. Each phase is a
+    new first_set_mask over caller-owned slabs; every sequence's logits follow the oracle run on
+    that sequence's own history (decisions stay fixed per sequence for its whole decode)."""
+    import torch
+    from paper_2410_12513_b200 import KVCache
+    shape, seed = fi.TINY, 31
+    L = shape.n_layers
+    w = fi.make_weights(shape, seed, False)
+    om = oracle_model(shape, w)
+    lens = [9, 14, 6, 11]
+    caps = [40, 40, 40, 40]
+    okv, gkv = synthetic_caches(shape, lens, caps, seed, False)
+    mask = fi.mask_bernoulli(4, L, 0.6, seed)
+    ctx = _ctx(shape, False, 4, 40, w)
+    logits = torch.empty((4, shape.vocab), dtype=torch.float32, device="cuda")
+
+    def steps(n, B, m, kvc, okv_, toks):
+        for _ in range(n):
+            ref = oracle.decode_step(om, toks, m, okv_)
+            ctx.decode_step(torch.from_numpy(toks).cuda(), kvc, logits[:B])
+            assert ctx.device_flags() == 0
+            err, agree = logits_check(logits[:B].cpu().numpy(), ref)
+            assert err.max() <= 1e-4 and agree.all()
+            toks = oracle.argmax(ref)
+        return toks
+
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = steps(2, 4, mask, gkv.c, okv, fi.tokens(shape, 4, seed, "first"))
+
+    # slot 1 finishes; a new sequence (prompt of 5 tokens, its own decisions) takes the slot
+    n_new = 5
+    new_row = fi.mask_bernoulli(1, L, 0.5, seed + 1)[0]
+    new_row[1] = 0
+    mask2 = mask.copy()
+    mask2[1] = new_row
+    for l in range(L):
+        kr = fi.synthetic_kv_rows(n_new, shape.kv_dim, seed + 2, f"k{l}", False)
+        vr = fi.synthetic_kv_rows(n_new, shape.kv_dim, seed + 2, f"v{l}", False)
+        ko, vo = okv.rows(l, 1)
+        ko[:], vo[:] = 0, 0
+        ko[:n_new], vo[:n_new] = kr, vr
+        gkv.load_rows(l, 1, kr, vr)
+    okv.len[:, 1] = n_new
+    okv.pos[1] = n_new
+    gkv.set_len(okv.len, okv.pos)
+    ctx.set_mask(torch.from_numpy(mask2).cuda())
+    toks = toks.copy()
+    toks[1] = fi.tokens(shape, 1, seed + 3, "new")[0]
+    toks = steps(2, 4, mask2, gkv.c, okv, toks)
+
+    # slot 3 finishes and is not refilled: the same slabs described as a batch of three
+    o3 = oracle.OracleKV(oracle.Shape(**shape.asdict()), caps[:3])
+    for l in range(L):
+        for b in range(3):
+            ks, vs = okv.rows(l, b)
+            kd, vd = o3.rows(l, b)
+            kd[:], vd[:] = ks, vs
+    o3.len[:] = okv.len[:, :3]
+    o3.pos[:] = okv.pos[:3]
+    len3 = gkv.len[:, :3].contiguous()
+    pos3 = gkv.pos[:3].contiguous()
+    kv3 = KVCache(gkv.k, gkv.v, gkv.slab_off[:3].contiguous(), gkv.slab_cap[:3].contiguous(), len3, pos3)
+    ctx.set_mask(torch.from_numpy(mask2[:3].copy()).cuda())
+    steps(2, 3, mask2[:3].copy(), kv3, o3, toks[:3].copy())
+    assert np.array_equal(len3.cpu().numpy(), o3.len) and np.array_equal(pos3.cpu().numpy(), o3.pos)
