@@ -76,6 +76,7 @@ def lib():
         _lib.fo_forward_full.restype = C.c_int
         _lib.fo_plan.restype = C.c_int
         _lib.fo_argmax.restype = C.c_int32
+        _lib.fo_sample_topk.restype = C.c_int32
     return _lib
 
 
@@ -267,6 +268,17 @@ def plan(mask):
 def argmax(logits):
     logits = np.ascontiguousarray(logits, dtype=np.float32)
     return np.array([lib().fo_argmax(_ptr(row), C.c_int32(row.shape[0])) for row in logits], dtype=np.int32)
+
+
+def sample_topk(logits_row, k, temperature, u):
+    """One row: -> (token, candidates[k] in order, probabilities[k])."""
+    row = np.ascontiguousarray(logits_row, dtype=np.float32)
+    cand = np.zeros(k, dtype=np.int32)
+    prob = np.zeros(k, dtype=np.float64)
+    t = lib().fo_sample_topk(_ptr(row), C.c_int32(row.shape[0]), C.c_int32(k), C.c_double(temperature),
+                             C.c_double(u), _ptr(cand), _ptr(prob))
+    _check(min(t, 0), "sample_topk")
+    return int(t), cand, prob
 
 
 def prefill(model: OracleModel, kv: OracleKV, b: int, tokens, want_router_in=True):

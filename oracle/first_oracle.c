@@ -385,6 +385,45 @@ int32_t fo_argmax(const float *v, int32_t n) {
     return best;
 }
 
+/* Temperature + top-k sampling of one row of logits (App. "Training and Inference Setup",
+ * inference settings: temperature 0.8, top-k over 10 tokens).  The candidates are the k largest
+ * logits, taken one by one (among equal values the lowest index first); their probabilities are
+ * the softmax of logit/T over the candidates only; the token is the first candidate, in that
+ * order, whose cumulative probability exceeds the uniform draw u in [0,1), which is an input.
+ * k = 1 or T = 0 is greedy decoding.  cand[k] and prob[k] (optional) receive the ordered
+ * candidates and their probabilities.  Returns the token, or FO_E_ARG. */
+int32_t fo_sample_topk(const float *v, int32_t n, int32_t k, double T, double u, int32_t *cand, double *prob) {
+    if (!v || n <= 0 || k <= 0 || k > n || T < 0.0 || !(u >= 0.0 && u < 1.0)) return FO_E_ARG;
+    int32_t *c = (int32_t *)malloc(sizeof(int32_t) * (size_t)k);
+    double *p = (double *)malloc(sizeof(double) * (size_t)k);
+    uint8_t *taken = (uint8_t *)calloc((size_t)n, 1);
+    if (!c || !p || !taken) { free(c); free(p); free(taken); return FO_E_ARG; }
+    for (int32_t j = 0; j < k; ++j) {
+        int32_t best = -1;
+        for (int32_t i = 0; i < n; ++i)
+            if (!taken[i] && (best < 0 || v[i] > v[best])) best = i;
+        taken[best] = 1;
+        c[j] = best;
+    }
+    int32_t token = c[0];
+    if (k == 1 || T == 0.0) {
+        for (int32_t j = 0; j < k; ++j) p[j] = j == 0 ? 1.0 : 0.0;
+    } else {
+        double sum = 0.0;
+        for (int32_t j = 0; j < k; ++j) { p[j] = exp(((double)v[c[j]] - (double)v[c[0]]) / T); sum += p[j]; }
+        double cum = 0.0;
+        token = c[k - 1];
+        for (int32_t j = 0; j < k; ++j) p[j] /= sum;
+        for (int32_t j = 0; j < k; ++j) {
+            cum += p[j];
+            if (u < cum) { token = c[j]; break; }
+        }
+    }
+    for (int32_t j = 0; j < k; ++j) { if (cand) cand[j] = c[j]; if (prob) prob[j] = p[j]; }
+    free(c); free(p); free(taken);
+    return token;
+}
+
 /* Active-row lists of a mask: for each layer the ascending sequence indices that keep
  * it (Sec. "Adaptive Router Module": one decision per sequence per layer). */
 int fo_plan(const uint8_t *mask, int32_t B, int32_t L, int32_t *idx, int32_t *cnt, int32_t *slot) {

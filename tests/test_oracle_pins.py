@@ -317,3 +317,59 @@ def test_bf16_cache_storage_rounds_once_like_torch():
     # ties round to even: 1 + 2^-8 is exactly between two bfloat16 values
     tie = np.array([[1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8]], np.float32)
     assert rnd(tie).tolist() == [[1.0, 1.015625]]
+
+
+# ------------------------------------------------------------------ sampling (temperature + top-k)
+def test_sampling_hand_worked_two_candidates():
+    """logits (1,3,2,0), k=2: candidates are tokens 1 then 2; at T=1 the first has probability
+    1/(1+e^-1) = 0.731059, at T=0.5 it has 1/(1+e^-2) = 0.880797 (worked by hand)."""
+    z = np.array([1.0, 3.0, 2.0, 0.0], np.float32)
+    t, cand, prob = oracle.sample_topk(z, 2, 1.0, 0.70)
+    assert list(cand) == [1, 2] and t == 1
+    assert abs(prob[0] - 0.7310585786) < 1e-9 and abs(prob.sum() - 1) < 1e-12
+    assert oracle.sample_topk(z, 2, 1.0, 0.74)[0] == 2
+    _, _, p = oracle.sample_topk(z, 2, 0.5, 0.0)
+    assert abs(p[0] - 0.8807970780) < 1e-9          # a lower temperature sharpens, not flattens
+    assert oracle.sample_topk(z, 2, 0.5, 0.87)[0] == 1 and oracle.sample_topk(z, 2, 0.5, 0.89)[0] == 2
+
+
+def test_sampling_reduces_to_greedy_and_to_plain_softmax_sampling():
+    g = np.random.default_rng(5)
+    z = g.normal(0, 2, 500).astype(np.float32)
+    for u in (0.0, 0.3, 0.999):
+        assert oracle.sample_topk(z, 1, 0.8, u)[0] == int(z.argmax())
+        assert oracle.sample_topk(z, 10, 0.0, u)[0] == int(z.argmax())
+    # k = n: inverse-CDF sampling from softmax(z/T) in descending order, by library routines
+    from scipy.special import softmax
+    order = np.argsort(-z.astype(np.float64), kind="stable")
+    cdf = np.cumsum(softmax(z.astype(np.float64)[order] / 0.8))
+    for u in g.random(200):
+        j = int(np.searchsorted(cdf, u, side="right"))
+        if abs(cdf[min(j, 499)] - u) < 1e-9 or (j and abs(cdf[j - 1] - u) < 1e-9):
+            continue
+        assert oracle.sample_topk(z, 500, 0.8, float(u))[0] == int(order[min(j, 499)])
+    _, cand, prob = oracle.sample_topk(z, 10, 0.8, 0.5)
+    assert list(cand) == list(order[:10])
+    assert np.allclose(prob, softmax(z.astype(np.float64)[order[:10]] / 0.8), atol=1e-12)
+
+
+def test_sampling_frequencies_and_ties():
+    """Over an even grid of draws each candidate is chosen in proportion to its probability;
+    equal logits enter in index order and share the mass equally; the rest is never chosen."""
+    z = np.array([0.5, 2.0, 2.0, -1.0, 2.0, 1.5], np.float32)
+    _, cand, prob = oracle.sample_topk(z, 4, 0.8, 0.0)
+    assert list(cand) == [1, 2, 4, 5]
+    assert prob[0] == prob[1] == prob[2] and abs(prob[3] / prob[0] - np.exp(-0.5 / 0.8)) < 1e-12
+    n = 4000
+    counts = np.zeros(6)
+    for i in range(n):
+        counts[oracle.sample_topk(z, 4, 0.8, (i + 0.5) / n)[0]] += 1
+    assert counts[0] == 0 and counts[3] == 0
+    assert np.abs(counts[cand] / n - prob).max() <= 1.0 / n + 1e-12
+
+
+def test_sampling_rejects_bad_arguments():
+    z = np.zeros(4, np.float32)
+    for k, T, u in ((0, 1.0, 0.5), (5, 1.0, 0.5), (2, -1.0, 0.5), (2, 1.0, 1.0), (2, 1.0, -0.1)):
+        with pytest.raises(RuntimeError):
+            oracle.sample_topk(z, k, T, u)
