@@ -203,7 +203,8 @@ int first_get_plan(first_ctx *ctx, int32_t *idx, int32_t *cnt, int32_t *slot);
  *   tokens        dev int32 [B]
  *   kv            host struct; see first_kv_cache
  *   logits        dev float32 [B][vocab], or NULL
- *   next_tokens   dev int32 [B] or NULL: argmax of the logits row, lowest index on ties
+ *   next_tokens   dev int32 [B] or NULL: argmax of the logits row, lowest index on ties (or a
+ *                 sampled token, see first_set_sampling)
  *   layer_inputs  dev float32 [n_layers][B][d_model] or NULL: the residual entering each
  *                 layer (what router l reads when prompts are prefilled token by token
  *                 with an all-keep mask)
@@ -212,6 +213,27 @@ int first_get_plan(first_ctx *ctx, int32_t *idx, int32_t *cnt, int32_t *slot);
  * slab or a bad token id. */
 int first_decode_step(first_ctx *ctx, const int32_t *tokens, const first_kv_cache *kv, float *logits,
                       int32_t *next_tokens, float *layer_inputs, void *stream);
+
+/* Next-token sampling with the paper's generation settings (appendix "Training and Inference
+ * Setup", inference settings: temperature 0.8, top-k sampling over 10 tokens).  Per row: the
+ * candidates are the top_k largest logits, equal values in index order; their weights are
+ * exp((logit - max) / temperature); the token is the first candidate, in that order, whose
+ * cumulative weight exceeds u * (sum of weights), u the row's uniform draw.  The draws are an
+ * input: the library holds no generator.  Arithmetic is float32.
+ *   logits     dev float32 [B][vocab]
+ *   top_k      1 .. FIRST_SAMPLE_TOPK_MAX (and <= vocab); 1 is greedy decoding
+ *   temperature >= 0; 0 is greedy decoding
+ *   uniforms   dev float32 [B], each in [0,1); a value outside selects the last candidate
+ *   tokens     dev int32 [B]
+ * first_sample_topk is stateless (no context; one launch on `stream`).
+ * first_set_sampling makes every later first_decode_step of the context fill next_tokens this
+ * way instead of by argmax, reading `uniforms` (borrowed; the caller refreshes its contents
+ * before each step, in stream order); top_k <= 1 or temperature 0 restores argmax.
+ * Errors: FIRST_E_ARG, FIRST_E_UNSUPPORTED (top_k > FIRST_SAMPLE_TOPK_MAX), FIRST_E_CUDA. */
+#define FIRST_SAMPLE_TOPK_MAX 16
+int first_set_sampling(first_ctx *ctx, int32_t top_k, float temperature, const float *uniforms);
+int first_sample_topk(const float *logits, int32_t B, int32_t vocab, int32_t top_k, float temperature,
+                      const float *uniforms, int32_t *tokens, void *stream);
 
 /* Wait for `stream`, read and clear the device flag word.  Returns FIRST_OK with
  * *flags = 0, or FIRST_E_DEVICE_FLAG with the FIRST_FLAG_* bits in *flags. */

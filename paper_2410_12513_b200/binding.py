@@ -72,6 +72,11 @@ def lib():
         L.first_launch_count.restype = C.c_int64
         L.first_launch_count.argtypes = [C.c_void_p]
         L.first_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int64]
+        L.first_set_sampling.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_void_p]
+        L.first_set_sampling.restype = C.c_int
+        L.first_sample_topk.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p,
+                                        C.c_void_p]
+        L.first_sample_topk.restype = C.c_int
         L.first_profile.argtypes = [C.c_void_p, C.c_int32]
         L.first_profile.restype = C.c_int
         L.first_profile_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -224,6 +229,26 @@ def first_set_option(h, name, value):
         raise FirstError(rc, "first_set_option")
 
 
+def first_set_sampling(h, top_k, temperature, uniforms):
+    """uniforms: CUDA float32 [B] (borrowed: refresh its contents before every step), or None with
+    top_k <= 1 / temperature 0 to go back to argmax."""
+    rc = lib().first_set_sampling(h, int(top_k), float(temperature), _dev(uniforms, torch.float32, "uniforms"))
+    if rc:
+        raise FirstError(rc, "first_set_sampling")
+
+
+def first_sample_topk(logits, top_k, temperature, uniforms, tokens, stream=None):
+    """logits CUDA float32 [B][vocab]; uniforms CUDA float32 [B]; tokens CUDA int32 [B] (output)."""
+    B, V = logits.shape
+    if uniforms.numel() != B or tokens.numel() != B:
+        raise ValueError("uniforms and tokens must have one entry per row of logits")
+    rc = lib().first_sample_topk(_dev(logits, torch.float32, "logits"), B, V, int(top_k), float(temperature),
+                                 _dev(uniforms, torch.float32, "uniforms"), _dev(tokens, torch.int32, "tokens"),
+                                 _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_sample_topk")
+
+
 def first_profile(h, enable):
     rc = lib().first_profile(h, int(bool(enable)))
     if rc:
@@ -282,6 +307,10 @@ class FirstContext:
 
     def set_option(self, name, value):
         first_set_option(self.h, name, value)
+
+    def set_sampling(self, top_k, temperature, uniforms):
+        self._uniforms = uniforms  # borrowed by the library until the next call
+        first_set_sampling(self.h, top_k, temperature, uniforms)
 
     def profile(self, enable):
         first_profile(self.h, enable)

@@ -97,6 +97,10 @@ struct first_ctx {
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
     int tc_mt2_min_rows = 1 << 30;
+    // sampling of the next token (greedy while sample_k <= 1)
+    int sample_k = 0;
+    float sample_inv_T = 1.f;
+    const float* sample_u = nullptr;
     int tc_ksplit_cap = 1;  // from this many active rows on, a projection CTA takes two weight tiles
 };
 
@@ -532,6 +536,9 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                               nullptr, false)))
             return rc;
     }
+    if (next_tokens && lg && c->sample_k > 1)
+        return launch_k(c, st, kClsStepEnd, step_end_sample, dim3(B), dim3(1024), 0, lg, V, c->sample_k, c->sample_inv_T,
+                        c->sample_u, next_tokens, kv->pos);
     return launch_k(c, st, kClsStepEnd, step_end, dim3(B), dim3(1024), 0, lg, V, next_tokens, kv->pos);
 }
 
@@ -802,6 +809,31 @@ int first_profile_read(first_ctx* c, int32_t n, double* ms, int64_t* launches, v
         launches[k] = k < kNumClasses ? c->prof_launches[k] : 0;
     }
     return FIRST_OK;
+}
+
+int first_set_sampling(first_ctx* c, int32_t top_k, float temperature, const float* uniforms) {
+    if (!c || top_k < 0 || !(temperature >= 0.f)) return FIRST_E_ARG;
+    if (top_k > FIRST_SAMPLE_TOPK_MAX) return FIRST_E_UNSUPPORTED;
+    if (top_k > c->d.vocab) return FIRST_E_ARG;
+    const bool greedy = top_k <= 1 || temperature == 0.f;
+    if (!greedy && !uniforms) return FIRST_E_ARG;
+    c->sample_k = greedy ? 0 : top_k;
+    c->sample_inv_T = greedy ? 1.f : 1.f / temperature;
+    c->sample_u = greedy ? nullptr : uniforms;
+    c->plan_version += 1;  // cached step graphs end in the previous choice of kernel and pointer
+    return FIRST_OK;
+}
+
+int first_sample_topk(const float* logits, int32_t B, int32_t vocab, int32_t top_k, float temperature,
+                      const float* uniforms, int32_t* tokens, void* stream) {
+    if (!logits || !uniforms || !tokens || B <= 0 || vocab <= 0 || top_k <= 0 || top_k > vocab || !(temperature >= 0.f))
+        return FIRST_E_ARG;
+    if (top_k > FIRST_SAMPLE_TOPK_MAX) return FIRST_E_UNSUPPORTED;
+    const bool greedy = top_k == 1 || temperature == 0.f;
+    step_end_sample<<<B, 1024, 0, static_cast<cudaStream_t>(stream)>>>(logits, vocab, greedy ? 1 : top_k,
+                                                                        greedy ? 1.f : 1.f / temperature, uniforms, tokens,
+                                                                        nullptr);
+    return cudaGetLastError() == cudaSuccess ? FIRST_OK : FIRST_E_CUDA;
 }
 
 int32_t first_kernel_class_count(void) { return kNumClasses; }

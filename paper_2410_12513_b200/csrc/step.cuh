@@ -237,4 +237,100 @@ __global__ void __launch_bounds__(1024) step_end(const float* __restrict__ logit
     if (threadIdx.x == 0) pos[b] += 1;
 }
 
+// End of a step with sampling: next token per row by temperature + top-k sampling (the paper's
+// inference settings, appendix on training and inference set-up).  The candidates are the k
+// largest logits (equal values: lowest index first); token = first candidate whose cumulative
+// softmax(logit / T) mass over the candidates exceeds the row's uniform draw u.  One block of
+// 1024 threads per row: every thread keeps the kSampleKMax best of the elements it reads, sorted,
+// in registers; k rounds of a block-wide argmax over the threads' list heads then pop the row's k
+// best in order; thread 0 walks the cumulative weights (u * sum < cum, so no division).
+constexpr int kSampleKMax = 16;
+
+__device__ __forceinline__ bool sample_before(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+
+__global__ void __launch_bounds__(1024) step_end_sample(const float* __restrict__ logits, int V, int k, float inv_T,
+                                                        const float* __restrict__ uniforms,
+                                                        int32_t* __restrict__ next, int32_t* __restrict__ pos) {
+    pdl_trigger();
+    pdl_wait();
+    const int b = blockIdx.x;
+    __shared__ float bv[2][32];
+    __shared__ int bi[2][32];
+    __shared__ float cand_v[kSampleKMax];
+    __shared__ int cand_i[kSampleKMax];
+    const float* row = logits + (size_t)b * V;
+    float tv[kSampleKMax];
+    int ti[kSampleKMax];
+#pragma unroll
+    for (int j = 0; j < kSampleKMax; ++j) { tv[j] = -INFINITY; ti[j] = 0x7fffffff; }
+    auto consider = [&](float v, int i) {
+        if (sample_before(v, i, tv[kSampleKMax - 1], ti[kSampleKMax - 1])) {
+            tv[kSampleKMax - 1] = v;
+            ti[kSampleKMax - 1] = i;
+#pragma unroll
+            for (int j = kSampleKMax - 1; j > 0; --j) {
+                if (sample_before(tv[j], ti[j], tv[j - 1], ti[j - 1])) {
+                    const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
+                    const int fi = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = fi;
+                }
+            }
+        }
+    };
+    if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0) {
+        const float4* r4 = reinterpret_cast<const float4*>(row);
+        for (int i = threadIdx.x; i < V / 4; i += 1024) {
+            const float4 v = r4[i];
+            consider(v.x, 4 * i); consider(v.y, 4 * i + 1); consider(v.z, 4 * i + 2); consider(v.w, 4 * i + 3);
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += 1024) consider(row[i], i);
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int r = 0; r < k; ++r) {
+        float best = tv[0];
+        int besti = ti[0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v = __shfl_xor_sync(0xffffffffu, best, o);
+            const int j = __shfl_xor_sync(0xffffffffu, besti, o);
+            if (sample_before(v, j, best, besti)) { best = v; besti = j; }
+        }
+        if (lane == 0) { bv[r & 1][warp] = best; bi[r & 1][warp] = besti; }
+        __syncthreads();
+        best = bv[r & 1][lane];
+        besti = bi[r & 1][lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v = __shfl_xor_sync(0xffffffffu, best, o);
+            const int j = __shfl_xor_sync(0xffffffffu, besti, o);
+            if (sample_before(v, j, best, besti)) { best = v; besti = j; }
+        }
+        if (threadIdx.x == 0) { cand_v[r] = best; cand_i[r] = besti; }
+        if (ti[0] == besti) {  // the owner of the winner moves on to its next best
+#pragma unroll
+            for (int j = 0; j + 1 < kSampleKMax; ++j) { tv[j] = tv[j + 1]; ti[j] = ti[j + 1]; }
+            tv[kSampleKMax - 1] = -INFINITY;
+            ti[kSampleKMax - 1] = 0x7fffffff;
+        }
+    }
+    if (threadIdx.x == 0) {
+        const float z0 = cand_v[0];
+        float sum = 0.f;
+        for (int j = 0; j < k; ++j) {
+            const float w = j == 0 ? 1.f : expf((cand_v[j] - z0) * inv_T);
+            cand_v[j] = w;
+            sum += w;
+        }
+        const float target = uniforms[b] * sum;
+        int pick = cand_i[k - 1];
+        float cum = 0.f;
+        for (int j = 0; j < k; ++j) {
+            cum += cand_v[j];
+            if (target < cum) { pick = cand_i[j]; break; }
+        }
+        next[b] = pick == 0x7fffffff ? 0 : pick;
+        if (pos) pos[b] += 1;
+    }
+}
+
 }  // namespace first

@@ -388,3 +388,98 @@ def test_batch_changes_between_steps():
     ctx.set_mask(torch.from_numpy(mask2[:3].copy()).cuda())
     steps(2, 3, mask2[:3].copy(), kv3, o3, toks[:3].copy())
     assert np.array_equal(len3.cpu().numpy(), o3.len) and np.array_equal(pos3.cpu().numpy(), o3.pos)
+
+
+# ------------------------------------------------------------------ sampling (temperature + top-k)
+def _sample_agrees(row, k, T, u, got):
+    """The oracle's token; where the draw sits within 1e-5 of a boundary of the oracle's cumulative
+    distribution (float32 on the device, float64 in the oracle) either neighbour is right."""
+    tok, cand, prob = oracle.sample_topk(row, k, T, u)
+    if got == tok:
+        return True
+    cdf = np.cumsum(prob)
+    j = list(cand).index(tok)
+    near = [cand[i] for i in (j - 1, j + 1) if 0 <= i < k and min(abs(cdf[min(i, j)] - u), 1) < 1e-5]
+    return got in near
+
+
+@pytest.mark.parametrize("V", [1000, 1003, 128256])
+def test_sample_topk_matches_oracle(V):
+    import torch
+    from paper_2410_12513_b200 import first_sample_topk
+    B = 6
+    g = np.random.default_rng(V)
+    logits = g.normal(0, 3, (B, V)).astype(np.float32)
+    logits[1] = np.round(logits[1] * 2) / 2          # many equal values: candidates enter in index order
+    logits[2, ::3] = -np.inf
+    logits[3] = 0.0                                    # all equal: the first k indices, equal shares
+    logits[4, V - 1] = 50.0                            # the last (tail) element wins
+    dl = torch.from_numpy(logits).cuda()
+    out = torch.empty(B, dtype=torch.int32, device="cuda")
+    for k, T in ((1, 0.8), (2, 0.8), (10, 0.8), (16, 1.7), (10, 0.0), (10, 0.05)):
+        for rep in range(6):
+            u = g.random(B).astype(np.float32)
+            if rep == 0:
+                u[:] = 0.0
+            first_sample_topk(dl, k, T, torch.from_numpy(u).cuda(), out)
+            got = out.cpu().numpy()
+            for b in range(B):
+                assert _sample_agrees(logits[b], k, T, float(u[b]), int(got[b])), (V, k, T, b, u[b], got[b])
+    # an even grid of draws visits every candidate of a row in proportion (coarse check of the whole table)
+    n = 512
+    rows = torch.from_numpy(np.repeat(logits[:1], n, 0)).cuda()
+    u = ((np.arange(n) + 0.5) / n).astype(np.float32)
+    outn = torch.empty(n, dtype=torch.int32, device="cuda")
+    first_sample_topk(rows, 10, 0.8, torch.from_numpy(u).cuda(), outn)
+    _, cand, prob = oracle.sample_topk(logits[0], 10, 0.8, 0.0)
+    counts = np.array([(outn.cpu().numpy() == c).sum() for c in cand])
+    assert counts.sum() == n and np.abs(counts / n - prob).max() <= 2.0 / n
+
+
+def test_sample_topk_rejects_bad_arguments():
+    import torch
+    from paper_2410_12513_b200 import FirstError, first_sample_topk
+    lg = torch.zeros((2, 64), device="cuda")
+    u = torch.zeros(2, device="cuda")
+    out = torch.empty(2, dtype=torch.int32, device="cuda")
+    for k, T in ((0, 1.0), (17, 1.0), (65, 1.0), (4, -1.0)):
+        with pytest.raises(FirstError):
+            first_sample_topk(lg, k, T, u, out)
+
+
+def test_decode_step_samples_when_asked():
+    """first_set_sampling switches the step's next-token kernel: the sampled tokens are the
+    oracle's sampling rule applied to the step's own logits (which are checked against the
+    oracle's as in every other case); switching back restores argmax."""
+    import torch
+    shape, seed, B = fi.TINY, 41, 5
+    w = fi.make_weights(shape, seed, False)
+    om = oracle_model(shape, w)
+    lens = fi.prompt_lengths(B, 1, 40, seed)
+    okv, gkv = synthetic_caches(shape, lens, [int(n) + 4 for n in lens], seed, False)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.6, seed)
+    ctx = _ctx(shape, False, B, int(max(lens)) + 4, w)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    u_dev = torch.zeros(B, dtype=torch.float32, device="cuda")
+    ctx.set_sampling(10, 0.8, u_dev)
+    logits = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda")
+    nxt = torch.empty(B, dtype=torch.int32, device="cuda")
+    toks = fi.tokens(shape, B, seed, "first")
+    g = np.random.default_rng(seed)
+    for step in range(3):
+        if step == 2:
+            ctx.set_sampling(0, 0.0, None)
+        u = g.random(B).astype(np.float32)
+        u_dev.copy_(torch.from_numpy(u))
+        ref = oracle.decode_step(om, toks, mask, okv)
+        ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits, nxt)
+        got, tok = logits.cpu().numpy(), nxt.cpu().numpy()
+        err, _ = logits_check(got, ref)
+        assert err.max() <= 1e-4
+        for b in range(B):
+            if step < 2:
+                assert _sample_agrees(got[b], 10, 0.8, float(u[b]), int(tok[b]))
+            else:
+                assert tok[b] == got[b].argmax()
+        toks = oracle.argmax(ref)
+    assert ctx.device_flags() == 0
