@@ -207,18 +207,26 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint
 
 constexpr int kTcSmemMax = 210 * 1024;
 
-// K ranges per weight tile for the reducing epilogues.  More ranges fill the SMs when a matrix has
-// few tiles, but every range adds m*n_out float32 reductions: keep that traffic below about half
-// of the weight bytes (ksplit <= K / (4 m)).
-int tc_ksplit(const first_ctx* c, int n_out, int K, int epi, int m) {
+// K ranges per weight tile for the reducing epilogues.  The CTAs of a projection should fill the
+// GPU's CTA slots (SMs x CTAs that fit per SM) in whole waves: among the counts allowed, take the
+// smallest whose last wave is nearly full.  Every range adds m*n_out float32 reductions: the count
+// is kept below K / (4 m), so that this traffic stays under about half of the weight bytes.
+int tc_ksplit(const first_ctx* c, int tiles, int K, int epi, int m, int slots) {
     if (epi == tc::kEpiStore || epi == tc::kEpiSwiglu) return 1;
-    m = std::min(m, 256);
-    const int mt = (m >= c->tc_mt2_min_rows) ? 2 : 1;
-    const int tiles = (n_out + tc::kBlockM * mt - 1) / (tc::kBlockM * mt), kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
-    int ks = (2 * c->n_sm + tiles / 2) / tiles;
-    ks = std::min(ks, kblocks / 4);
-    if (c->tc_ksplit_cap) ks = std::min(ks, std::max(1, K / (4 * std::max(m, 1))));
-    return std::max(1, ks);
+    const int kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+    int cap = std::max(1, kblocks / 4);
+    if (c->tc_ksplit_cap) cap = std::min(cap, std::max(1, K / (4 * std::max(std::min(m, 256), 1))));
+    cap = std::min(cap, std::max(1, (2 * slots + tiles - 1) / tiles));  // never more than two waves' worth
+    double best_eff = 0.0;
+    for (int ks = 1; ks <= cap; ++ks) {
+        const int units = tiles * ks, waves = (units + slots - 1) / slots;
+        best_eff = std::max(best_eff, (double)units / ((double)waves * slots));
+    }
+    for (int ks = 1; ks <= cap; ++ks) {
+        const int units = tiles * ks, waves = (units + slots - 1) / slots;
+        if ((double)units / ((double)waves * slots) >= 0.97 * best_eff) return ks;
+    }
+    return 1;
 }
 
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
@@ -241,13 +249,13 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.pair_rows = c->pair_rows;
         const int tile_rows = epi == tc::kEpiSwiglu ? (p.mt == 1 ? c->pair_rows : 128) : tc::kBlockM * p.mt;
         const int tiles = (n_out + tile_rows - 1) / tile_rows;
-        p.ksplit = tc_ksplit(c, n_out, K, epi, mm);
         p.act = act ? act + (size_t)r0 * n_out : nullptr;
         p.act_hi = act_hi ? act_hi + (size_t)r0 * n_out : nullptr;
         p.act_lo = act_lo ? act_lo + (size_t)r0 * n_out : nullptr;
         const int stage_bytes = tc::kABytes * p.mt + p.n_pad * 128 * (p.use_lo ? 2 : 1);
         const int budget = (3 * stage_bytes <= c->tc_smem_kb * 1024) ? c->tc_smem_kb * 1024 : 200 * 1024;
         p.stages = std::max(1, std::min(8, budget / stage_bytes));
+        p.ksplit = tc_ksplit(c, tiles, K, epi, mm, c->n_sm * (budget == c->tc_smem_kb * 1024 ? 2 : 1));
         int cols = 32;
         while (cols < p.n_pad) cols *= 2;
         p.acc_cols = cols;
@@ -273,7 +281,7 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
                     : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
                     : e == tc::kEpiSwiglu ? tc::gemm_tc_kernel<tc::kEpiSwiglu>
                                           : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
-        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(192), smem, tmA, tmA2, tmBh, tmBl, p))) return rc;
+        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(320), smem, tmA, tmA2, tmBh, tmBl, p))) return rc;
     }
     return FIRST_OK;
 }
@@ -476,9 +484,9 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         float* f32 = t ? nullptr : c->xn;
         __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
         // split-K projections reduce into float32 accumulators that the preceding norm kernel clears
-        const bool zero_qkv = t && tc_ksplit(c, c->qkvd, D, tc::kEpiAtomic, m) > 1;
+        const bool zero_qkv = t;  // (cleared even when a projection ends up with one K range and plain stores)
         const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
-        const bool zero_gu = t && !fused_ffn && tc_ksplit(c, 2 * F, D, tc::kEpiAtomic, m) > 1;
+        const bool zero_gu = t && !fused_ffn;
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))

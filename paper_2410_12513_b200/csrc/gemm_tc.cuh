@@ -13,8 +13,8 @@
 // The gate/up projection has its own epilogue: its tile is 64 gate rows stacked on the matching
 // 64 up rows (two TMA boxes), the whole K range in one CTA, and the epilogue applies
 // silu(gate)*up in registers and writes the activation (and its hi/lo split) directly.
-// Roles inside a CTA of 6 warps: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2..5 = epilogue (one TMEM lane quadrant each).  Every wait is bounded.
+// Roles inside a CTA of 10 warps: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..9 = epilogue (two per TMEM lane quadrant, alternate 16-column chunks).  Every wait is bounded.
 #pragma once
 #include <cuda.h>
 
@@ -127,7 +127,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 
 // Dynamic shared memory: [stages][A mt*16 KB | B_hi n_pad*128 | B_lo n_pad*128] (1024-aligned), then barriers.
 template <int EPI>
-__global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+__global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                       const __grid_constant__ CUtensorMap tmA2,
                                                       const __grid_constant__ CUtensorMap tmBh,
                                                       const __grid_constant__ CUtensorMap tmBl, const GemmParams p) {
@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     const uint32_t tmem_full_bar = bars + 16u * p.stages;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ int idx_s[256];  // active-row list of the scattering epilogue
 
     pdl_trigger();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -248,16 +249,23 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             umma_commit(tmem_full_bar);  // accumulator complete (arrives even after a failed wait)
         }
     } else {
+        // Epilogue: 8 warps.  Warp w reads TMEM lanes 32*(w%4) .. +31 (its quadrant); the two warps of a
+        // quadrant take alternate 16-column chunks of the accumulator.
+        const int quad = warp & 3, half = (warp - 2) >> 2;
         pdl_wait();  // the epilogue reads idx and reduces into buffers the previous kernels own
+        if (EPI == kEpiScatterAtomic) {
+            for (int e = (int)threadIdx.x - 64; e < p.m; e += 256) idx_s[e] = p.idx[e];
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const bool run = ok && nkb > 0;
         if (EPI == kEpiSwiglu && p.mt == 2) {
             // accumulator 0 = 128 gate features, accumulator 1 = the same 128 up features: no exchange needed
-            const int quad = warp & 3;
             const int f = tile * 128 + quad * 32 + lane;
             const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
-            if (ok && nkb > 0) {
-                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+            if (run) {
+                for (int c0 = half * 16; c0 < p.n_pad; c0 += 32) {
                     uint32_t vg[16], vu[16];
                     tmem_ld16(lane_addr + (uint32_t)c0, vg);
                     tmem_ld16(lane_addr + (uint32_t)(p.acc_cols + c0), vu);
@@ -281,56 +289,50 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 }
             }
         } else if (EPI == kEpiSwiglu) {
-            // lanes [0, R) of the accumulator hold gate features, lanes [R, 2R) the matching up features
-            // (R = pair_rows; lanes from 2R up saw stale shared memory and are ignored).  Up lanes park
-            // their values in shared memory (the ring is idle once the accumulator is complete), gate
-            // lanes combine.  u_s[j][feature]: conflict-free both ways.
-            const int quad = warp & 3, R = p.pair_rows;
-            float* u_s = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)));
+            // Lanes [0, R) of the accumulator hold gate features, lanes [R, 2R) the matching up features
+            // (R = pair_rows; lanes from 2R up saw stale shared memory and are ignored).  Per 16-column
+            // chunk every lane loads its values once; up lanes park theirs in a small double buffer in
+            // shared memory (the ring is idle once the accumulator is complete), the four warps of this
+            // half meet at a named barrier, and gate lanes combine.  u[column][feature]: conflict-free.
+            const int R = p.pair_rows;
+            float* u_s = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw))) + half * (2 * 16 * 64);
             const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16);
-            const bool run = ok && nkb > 0;
             const int gl = quad * 32 + lane;  // accumulator lane of this thread
-            if (run && quad * 32 + 31 >= R && quad * 32 < 2 * R) {  // this warp holds some up lanes
-                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(lane_addr + (uint32_t)c0, v);
-                    if (gl >= R && gl < 2 * R) {
+            const int f = tile * R + gl;
+            int k = 0;
+            for (int c0 = half * 16; c0 < p.n_pad; c0 += 32, ++k) {  // every thread of the half takes every trip
+                uint32_t v[16];
+                tmem_ld16(lane_addr + (uint32_t)c0, v);
+                float* ub = u_s + (k & 1) * (16 * 64);
+                if (gl >= R && gl < 2 * R) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) u_s[(c0 + c) * 64 + (gl - R)] = __uint_as_float(v[c]);
-                    }
+                    for (int c = 0; c < 16; ++c) ub[c * 64 + (gl - R)] = __uint_as_float(v[c]);
                 }
-            }
-            asm volatile("bar.sync 2, 128;" ::: "memory");
-            if (run && quad * 32 < R) {  // this warp holds some gate lanes
-                const int f = tile * R + gl;
-                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(lane_addr + (uint32_t)c0, v);
-                    if (gl < R && f < p.n_out) {
+                if (half == 0) asm volatile("bar.sync 2, 128;" ::: "memory");
+                else asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (run && gl < R && f < p.n_out) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int j = c0 + c;
-                            if (j < p.m) {
-                                const float g = __uint_as_float(v[c]);
-                                const float y = g / (1.f + expf(-g)) * u_s[j * 64 + gl];
-                                const size_t o = (size_t)j * p.n_out + f;
-                                if (p.act) p.act[o] = y;
-                                if (p.act_hi) {
-                                    const __nv_bfloat16 h = __float2bfloat16_rn(y);
-                                    p.act_hi[o] = h;
-                                    p.act_lo[o] = __float2bfloat16_rn(y - __bfloat162float(h));
-                                }
+                    for (int c = 0; c < 16; ++c) {
+                        const int j = c0 + c;
+                        if (j < p.m) {
+                            const float g = __uint_as_float(v[c]);
+                            const float y = g / (1.f + expf(-g)) * ub[c * 64 + gl];
+                            const size_t o = (size_t)j * p.n_out + f;
+                            if (p.act) p.act[o] = y;
+                            if (p.act_hi) {
+                                const __nv_bfloat16 h = __float2bfloat16_rn(y);
+                                p.act_hi[o] = h;
+                                p.act_lo[o] = __float2bfloat16_rn(y - __bfloat162float(h));
                             }
                         }
                     }
                 }
             }
-        } else if (ok && nkb > 0) {
-            const int quad = warp & 3;
+        } else if (run) {
             for (int a = 0; a < p.mt; ++a) {
                 const int f = (tile * p.mt + a) * kBlockM + quad * 32 + lane;
                 const uint32_t lane_addr = tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * p.acc_cols);
-                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                for (int c0 = half * 16; c0 < p.n_pad; c0 += 32) {
                     uint32_t v[16];
                     tmem_ld16(lane_addr + (uint32_t)c0, v);
                     if (f < p.n_out) {
@@ -341,7 +343,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                                 const float val = __uint_as_float(v[c]);
                                 if (EPI == kEpiStore) p.Y[(size_t)j * p.ldy + f] = val;
                                 else if (EPI == kEpiAtomic) atomicAdd(p.Y + (size_t)j * p.ldy + f, val);
-                                else atomicAdd(p.Y + (size_t)p.idx[j] * p.ldy + f, val);
+                                else atomicAdd(p.Y + (size_t)idx_s[j] * p.ldy + f, val);
                             }
                         }
                     }
