@@ -274,6 +274,9 @@ const char *first_kernel_class_name(int32_t k);
  *                    activation tile (default: never)
  *   "tc_ksplit_cap"  0 = do not bound the number of K ranges by the reduction traffic
  *   "tc_smem_kb"     shared-memory budget per projection CTA when two CTAs per SM are wanted (110)
+ *   "fuse_rope"      0 = a separate kernel rotates q/k and appends the new key/value before attention.
+ *                    Default 1: the tuned attention kernel (bfloat16 caches, head_dim 64/128) does both
+ *                    itself, from the QKV projection's output.
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
  *                    its epilogue (needs ffn_dim % 64 == 0).

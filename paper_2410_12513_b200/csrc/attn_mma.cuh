@@ -47,10 +47,24 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 }
 __device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// When qkv is set the kernel works straight from the QKV projection's output
+// ([m][(Hq+2*Hkv)*HD] float32: q heads, k heads, v heads): it rotates and scales q itself, and the
+// CTA that holds a row's last chunk rotates the new token's key, rounds key and value to bfloat16,
+// writes them at the end of the row's slab and drops them into its shared-memory tile, so that no
+// separate rotate-and-append kernel runs.  cs: [B][HD/2] (cos, sin) of each sequence's position.
+struct RopeFuse {
+    const float* qkv;
+    const float2* cs;
+    float qscale;
+    __nv_bfloat16* k_slab;  // this layer's [Hkv][cap_total][HD]
+    __nv_bfloat16* v_slab;
+};
+
 // grid (S_max, Hkv, m), 160 threads.  Work item = (active row i, kv head h, chunk c):
-// tokens [c*C, min(T, (c+1)*C)), T = len[b]+1 (the new token was just written at row len[b];
-// T = len[b] if the slab was full and nothing was written), taken from rowinfo[i].  Chunks past T exit at once.
-// q: [m][Hq][HD] float32, pre-scaled by 1/sqrt(HD).  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64x64.
+// tokens [c*C, min(T, (c+1)*C)), T = len[b]+1 (the new token sits at row len[b]: already written by the
+// rotate-and-append kernel, or put there by this kernel, see RopeFuse; T = len[b] if the slab was full
+// and nothing is written), taken from rowinfo[i].  Chunks past T exit at once.
+// q: [m][Hq][HD] float32, pre-scaled by 1/sqrt(HD) (unused with RopeFuse).  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64x64.
 // Scratch: o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum),
 // ticket [m][Hkv] (zero between launches: the merging CTA resets it).
 // Output: out [m][Hq*HD] float32 and/or its bfloat16 hi/lo split (either may be NULL).
@@ -63,7 +77,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                                                       uint32_t* __restrict__ ticket, float* __restrict__ out,
                                                       __nv_bfloat16* __restrict__ out_hi,
                                                       __nv_bfloat16* __restrict__ out_lo,
-                                                      uint32_t* __restrict__ flags) {
+                                                      uint32_t* __restrict__ flags, const RopeFuse rf) {
     constexpr int kHalves = HD / 64;              // 128-byte column groups per row
     constexpr int kBox = kTile * 128;             // bytes of one 64-token x 64-element box
     constexpr int kStageBytes = 2 * kHalves * kBox;
@@ -73,8 +87,12 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     pdl_trigger();
     pdl_wait();
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
-    const longlong2 ri = rowinfo[i];  // (tokens present incl. the new one, first slab row), written by rope_append
-    const int T = (int)ri.x;
+    // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
+    const longlong2 ri = rowinfo[i];
+    const int T = (int)(ri.x & 0xffffffffll);
+    const int brow = (int)(ri.x >> 32);
+    const int64_t slab0 = ri.y & ((1ll << 62) - 1);
+    const bool append = rf.qkv != nullptr && (ri.y >> 62) != 0;
     const int t_begin = c * C;
     if (t_begin >= T) return;
     const int n_chunks = (T + C - 1) / C;
@@ -100,7 +118,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
 
     if (warp == 4) {  // ---------------- producer
         if (lane == 0) {
-            const int64_t row0 = (int64_t)h * cap_total + ri.y + t_begin;
+            const int64_t row0 = (int64_t)h * cap_total + slab0 + t_begin;
             uint64_t pol;  // cached keys/values are read once per step: do not let them displace L2 contents
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
             int issued = 0;
@@ -130,7 +148,30 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     // ---------------- consumers: warp w owns tokens [16w, 16w+16) of every tile
     const int g = lane >> 2, tq = lane & 3;
     uint32_t qh[kKSteps][2], ql[kKSteps][2];  // A fragments: (k0..k0+1), (k0+8..k0+9) of row g
-    {
+    const int qkv_stride = (Hq + 2 * (int)gridDim.y) * HD;
+    const float2* csr = rf.cs + (size_t)brow * (HD / 2);
+    if (rf.qkv) {
+        constexpr int kHalf = HD / 2;
+        const float* qrow = rf.qkv + (size_t)i * qkv_stride + ((size_t)h * G + (g < G ? g : 0)) * HD;
+        auto rot2 = [&](int dd) {  // rotated, scaled q[dd], q[dd+1] (dd even; both on the same side of HD/2)
+            const int lo_d = dd < kHalf ? dd : dd - kHalf;
+            const float2 a = *reinterpret_cast<const float2*>(qrow + lo_d);
+            const float2 bb = *reinterpret_cast<const float2*>(qrow + lo_d + kHalf);
+            const float4 cc = *reinterpret_cast<const float4*>(csr + lo_d);  // cos, sin of lo_d and lo_d + 1
+            return dd < kHalf ? make_float2((a.x * cc.x - bb.x * cc.y) * rf.qscale, (a.y * cc.z - bb.y * cc.w) * rf.qscale)
+                              : make_float2((bb.x * cc.x + a.x * cc.y) * rf.qscale, (bb.y * cc.z + a.y * cc.w) * rf.qscale);
+        };
+#pragma unroll
+        for (int ks = 0; ks < kKSteps; ++ks) {
+            float2 v0 = make_float2(0.f, 0.f), v1 = v0;
+            if (g < G) {
+                v0 = rot2(ks * 16 + 2 * tq);
+                v1 = rot2(ks * 16 + 8 + 2 * tq);
+            }
+            split2(v0.x, v0.y, qh[ks][0], ql[ks][0]);
+            split2(v1.x, v1.y, qh[ks][1], ql[ks][1]);
+        }
+    } else {
         const float* qrow = q + ((size_t)i * Hq + (size_t)h * G + (g < G ? g : 0)) * HD;
 #pragma unroll
         for (int ks = 0; ks < kKSteps; ++ks) {
@@ -166,6 +207,37 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                     *reinterpret_cast<uint4*>(vptr + (cc >> 3) * kBox + row * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
             }
             __syncwarp();
+        }
+        if (append && t_end == T && j == n_tiles - 1) {
+            // The new token (row T-1 of the sequence) is the last row of this tile: what TMA fetched for
+            // it is whatever the slab held.  The warp that owns the row builds the key and value from
+            // the projection output, stores them in the slab for later steps and in the tile for this one.
+            const int r = (T - 1) - tile_t0;
+            if ((r >> 4) == warp) {
+                constexpr int kHalf = HD / 2;
+                const float* krow = rf.qkv + (size_t)i * qkv_stride + (size_t)Hq * HD + (size_t)h * HD;
+                const float* vrow = krow + (size_t)gridDim.y * HD;
+                uint8_t* kst = base_ptr + (size_t)s * kStageBytes;
+                uint8_t* vst = kst + kHalves * kBox;
+                const size_t grow = ((size_t)h * cap_total + (size_t)slab0 + (size_t)(T - 1)) * HD;
+                auto put = [&](uint8_t* st, __nv_bfloat16* slab, int dd, __nv_bfloat162 val) {
+                    const int cc = (dd & 63) >> 3;
+                    *reinterpret_cast<__nv_bfloat162*>(st + (dd >> 6) * kBox + r * 128 + ((cc ^ (r & 7)) << 4) + (dd & 7) * 2) = val;
+                    *reinterpret_cast<__nv_bfloat162*>(slab + grow + dd) = val;
+                };
+                for (int pp = 2 * lane; pp < kHalf; pp += 64) {
+                    const float2 a = *reinterpret_cast<const float2*>(krow + pp);
+                    const float2 bb = *reinterpret_cast<const float2*>(krow + pp + kHalf);
+                    const float4 cc = *reinterpret_cast<const float4*>(csr + pp);
+                    put(kst, rf.k_slab, pp, __floats2bfloat162_rn(a.x * cc.x - bb.x * cc.y, a.y * cc.z - bb.y * cc.w));
+                    put(kst, rf.k_slab, pp + kHalf, __floats2bfloat162_rn(bb.x * cc.x + a.x * cc.y, bb.y * cc.z + a.y * cc.w));
+                    const float2 va = *reinterpret_cast<const float2*>(vrow + pp);
+                    const float2 vb = *reinterpret_cast<const float2*>(vrow + pp + kHalf);
+                    put(vst, rf.v_slab, pp, __floats2bfloat162_rn(va.x, va.y));
+                    put(vst, rf.v_slab, pp + kHalf, __floats2bfloat162_rn(vb.x, vb.y));
+                }
+                __syncwarp();
+            }
         }
         // ---- scores S[g][token] for this warp's 16 tokens (two n-tiles of 8)
         float sc[2][4];

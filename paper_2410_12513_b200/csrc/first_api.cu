@@ -93,6 +93,7 @@ struct first_ctx {
     int attn_simple = -1;
     int tc_use_lo = 1;
     int fuse_swiglu = 1;
+    int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
@@ -378,12 +379,20 @@ int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorM
 
 template <int HD, int G>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
-                       const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx, int C, float* out,
-                       __nv_bfloat16* out_hi, __nv_bfloat16* out_lo) {
+                       const first_kv_cache* kv, const void* kc, const void* vc, int C, float* out,
+                       __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
+    attn::RopeFuse rf{};
+    if (fuse_rope) {
+        rf.qkv = c->qkv;
+        rf.cs = c->cs;
+        rf.qscale = qscale;
+        rf.k_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(kc));
+        rf.v_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(vc));
+    }
     return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
                     c->rowinfo, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
-                    out_hi, out_lo, c->flags);
+                    out_hi, out_lo, c->flags, rf);
 }
 
 template <int HD, int G>
@@ -406,7 +415,7 @@ int attn_mma_setup(first_ctx* c) {
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const first_kv_cache* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
-                    __nv_bfloat16* out_lo) {
+                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -426,7 +435,7 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     dim3 grid(S, d.n_kv_heads, m);
 #define FIRST_ATTN_MMA(HD, G)                 \
     if (d.head_dim == HD && c->group == G)    \
-        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, len_l, idx, C, out, out_hi, out_lo);
+        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale);
     FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 3) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
     FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 3) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
@@ -469,6 +478,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const float qscale = 1.0f / std::sqrt((float)hd);
     const int norm_threads = std::max(32, std::min(1024, (D / 4 + 31) / 32 * 32));  // one float4 per thread when the row allows
     const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
+    const bool fuse_rope = mma_attn && c->fuse_rope;
 
     for (int l = 0; l < L; ++l) {
         if (layer_inputs) {
@@ -489,18 +499,25 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool zero_gu = t && !fused_ffn;
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
-                           d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, nullptr, nullptr)))
+                           d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, static_cast<int32_t*>(nullptr),
+                           fuse_rope ? kv->slab_cap : nullptr, fuse_rope ? c->rowinfo : nullptr,
+                           fuse_rope ? static_cast<const int32_t*>(len_l) : nullptr, fuse_rope ? kv->slab_off : nullptr,
+                           c->flags)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
                               c->qkv, c->qkvd, nullptr, true, zero_qkv)))
             return rc;
-        if ((rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
+        // The tuned attention kernel rotates q itself and appends the new token's key and value (its
+        // row facts come from the norm kernel above); the general path has a kernel for that.
+        if (!fuse_rope &&
+            (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
                            0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total, kv->slab_off,
                            kv->slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr)))
             return rc;
         if (mma_attn) {
-            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, t ? nullptr : c->att, xh, xl)))
+            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, t ? nullptr : c->att, xh, xl,
+                                      fuse_rope, qscale)))
                 return rc;
         } else {
             if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
@@ -513,7 +530,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             return rc;
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->ffn_norm[l],
-                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap)))
+                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
@@ -538,7 +555,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool t = tc_for(B);
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, D, c->final_norm,
                            d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
-                           nullptr)))
+                           nullptr, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
             return rc;
         if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
                               nullptr, false)))
@@ -856,6 +873,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "use_graph")) c->use_graph = value != 0;
     else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
+    else if (!std::strcmp(name, "fuse_rope")) c->fuse_rope = value != 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;

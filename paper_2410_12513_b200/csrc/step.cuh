@@ -57,11 +57,19 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 //   zero_row: row i of a float32 accumulator (zero_cols wide) is cleared for a split-K projection;
 //   len_inc:  the row's cache length is advanced by one (unless its slab is full) -- done here,
 //             after the layer's attention, so no attention block can see a half-updated length.
+//   rowinfo:  (attention side) what the attention kernel needs to know about row i, in one 16-byte
+//             word: x = tokens to attend over (cache length + the new token, at most the slab's
+//             capacity) | batch row << 32;  y = first slab row | (1 << 62 when the new token's key
+//             and value are to be appended).  A full slab raises FIRST_FLAG_KV_FULL.
 __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
                                                      const float* __restrict__ gain, float eps, float* __restrict__ out,
                                                      __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                      float* __restrict__ zero_row, int zero_cols,
-                                                     int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap) {
+                                                     int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap,
+                                                     longlong2* __restrict__ rowinfo,
+                                                     const int32_t* __restrict__ len_ro,
+                                                     const int64_t* __restrict__ slab_off,
+                                                     uint32_t* __restrict__ flags) {
     // One pass: the row stays in registers between the sum of squares and the scaling
     // (up to kMaxV float4 per thread; longer rows re-read the tail from L1/L2).
     constexpr int kMaxV = 4;
@@ -80,6 +88,13 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x
     if (len_inc && threadIdx.x == 0) {
         const int T = len_inc[b];
         if (T < slab_cap[b]) len_inc[b] = T + 1;
+    }
+    if (rowinfo && threadIdx.x == (blockDim.x > 32 ? 32 : 0)) {
+        const int T = len_ro[b], cap = slab_cap[b];
+        const bool room = T < cap;
+        rowinfo[i] = make_longlong2((long long)min(T + 1, cap) | ((long long)b << 32),
+                                    (long long)slab_off[b] | (room ? (1ll << 62) : 0ll));
+        if (!room) atomicOr(flags, FIRST_FLAG_KV_FULL);
     }
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)b * D);
     float4 r[kMaxV];
@@ -139,7 +154,7 @@ __global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv,
     pdl_wait();
     const int i = blockIdx.y, head = blockIdx.x, d = threadIdx.x, b = idx[i];
     if (rowinfo && head == 0 && d == 0)  // what attention needs to know about this row, in one 16-byte word
-        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]), (long long)slab_off[b]);
+        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]) | ((long long)b << 32), (long long)slab_off[b]);
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
     const float* row = qkv + (size_t)i * (qd + 2 * kvd) + (size_t)head * hd;

@@ -183,6 +183,7 @@ def test_decode_bf16_gemv_path_and_general_attention_by_option():
     mask = fi.mask_bernoulli(5, shape.n_layers, 0.7, 24)
     _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"max_gemv_rows": 8, "attn_simple": 1})
     _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"fuse_swiglu": 0, "use_pdl": 0, "use_graph": 0})
+    _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"fuse_rope": 0})
 
 
 def test_all_skip_and_all_keep_masks():
