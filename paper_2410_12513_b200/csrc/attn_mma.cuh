@@ -93,10 +93,14 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     const int brow = (int)(ri.x >> 32);
     const int64_t slab0 = ri.y & ((1ll << 62) - 1);
     const bool append = rf.qkv != nullptr && (ri.y >> 62) != 0;
-    const int t_begin = c * C;
-    if (t_begin >= T) return;
+    // A row of T tokens is cut into ceil(T / C) chunks of equal length (a multiple of the tile), not
+    // into full chunks plus a short remainder: its CTAs then finish together.
     const int n_chunks = (T + C - 1) / C;
-    const int t_end = min(T, t_begin + C);
+    if (c >= n_chunks) return;
+    const int Cb = ((T + n_chunks - 1) / n_chunks + kTile - 1) / kTile * kTile;
+    const int t_begin = c * Cb;
+    if (t_begin >= T) return;  // (cannot happen: (n_chunks - 1) * Cb < T)
+    const int t_end = min(T, t_begin + Cb);
     const int n_tiles = (t_end - t_begin + kTile - 1) / kTile;
 
     extern __shared__ uint8_t smem_raw[];

@@ -422,9 +422,11 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     if (C <= 0) {
         const double est = 0.6 * (double)m * d.n_kv_heads * d.max_tokens_per_seq;
         C = (int)(est / (4.0 * c->n_sm));
-        C = std::max(512, std::min(2048, C));
+        C = std::max(1024, std::min(2048, C));
         // few rows: smaller chunks until there is at least one work item per SM
         while (C > 128 && est / C < c->n_sm) C /= 2;
+        // many rows: whole rows already fill the CTA slots several times over, and an unsplit row needs no merge
+        if (m * d.n_kv_heads >= 3 * c->n_sm && d.max_tokens_per_seq <= 2048) C = d.max_tokens_per_seq;
     }
     C = std::max(C, (d.max_tokens_per_seq + c->max_splits - 1) / c->max_splits);
     C = (C + attn::kTile - 1) / attn::kTile * attn::kTile;
