@@ -252,11 +252,11 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
         // Epilogue: 8 warps.  Warp w reads TMEM lanes 32*(w%4) .. +31 (its quadrant); the two warps of a
         // quadrant take alternate 16-column chunks of the accumulator.
         const int quad = warp & 3, half = (warp - 2) >> 2;
-        pdl_wait();  // the epilogue reads idx and reduces into buffers the previous kernels own
-        if (EPI == kEpiScatterAtomic) {
+        if (EPI == kEpiScatterAtomic) {  // the active-row list is fixed between first_set_mask calls
             for (int e = (int)threadIdx.x - 64; e < p.m; e += 256) idx_s[e] = p.idx[e];
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
+        pdl_wait();  // the epilogue reduces into buffers the previous kernels own
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const bool run = ok && nkb > 0;

@@ -82,9 +82,9 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x
         const int k = threadIdx.x + v * nt;
         if (k < nv) g[v] = __ldg(reinterpret_cast<const float4*>(gain) + k);
     }
+    const int b = idx ? idx[i] : i;  // the plan is fixed between first_set_mask calls: no need to wait for it
     pdl_wait();
     __shared__ float red[32];
-    const int b = idx ? idx[i] : i;
     if (len_inc && threadIdx.x == 0) {
         const int T = len_inc[b];
         if (T < slab_cap[b]) len_inc[b] = T + 1;
