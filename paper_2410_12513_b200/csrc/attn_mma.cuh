@@ -71,8 +71,8 @@ struct RopeFuse {
 template <int HD, int G>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
-                                                      const float* __restrict__ q, int64_t cap_total,
-                                                      const longlong2* __restrict__ rowinfo, int Hq, int C,
+                                                      const float* q, int64_t cap_total,
+                                                      const longlong2* rowinfo, int Hq, int C,
                                                       float* __restrict__ o_part, float2* __restrict__ ml_part,
                                                       uint32_t* __restrict__ ticket, float* __restrict__ out,
                                                       __nv_bfloat16* __restrict__ out_hi,
@@ -85,24 +85,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     static_assert(G <= 8, "query heads of a group are the 8 hi rows of the A fragment");
 
     pdl_trigger();
-    pdl_wait();
-    const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
-    // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
-    const longlong2 ri = rowinfo[i];
-    const int T = (int)(ri.x & 0xffffffffll);
-    const int brow = (int)(ri.x >> 32);
-    const int64_t slab0 = ri.y & ((1ll << 62) - 1);
-    const bool append = rf.qkv != nullptr && (ri.y >> 62) != 0;
-    // A row of T tokens is cut into ceil(T / C) chunks of equal length (a multiple of the tile), not
-    // into full chunks plus a short remainder: its CTAs then finish together.
-    const int n_chunks = (T + C - 1) / C;
-    if (c >= n_chunks) return;
-    const int Cb = ((T + n_chunks - 1) / n_chunks + kTile - 1) / kTile * kTile;
-    const int t_begin = c * Cb;
-    if (t_begin >= T) return;  // (cannot happen: (n_chunks - 1) * Cb < T)
-    const int t_end = min(T, t_begin + Cb);
-    const int n_tiles = (t_end - t_begin + kTile - 1) / kTile;
-
+    // Set-up that needs nothing from the previous kernel comes first, so that it overlaps that kernel's tail.
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - tc::smem_u32(smem_raw));
@@ -119,6 +102,24 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait();
+    const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
+    // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
+    const longlong2 ri = __ldcg(&rowinfo[i]);
+    const int T = (int)(ri.x & 0xffffffffll);
+    const int brow = (int)(ri.x >> 32);
+    const int64_t slab0 = ri.y & ((1ll << 62) - 1);
+    const bool append = rf.qkv != nullptr && (ri.y >> 62) != 0;
+    // A row of T tokens is cut into ceil(T / C) chunks of equal length (a multiple of the tile), not
+    // into full chunks plus a short remainder: its CTAs then finish together.
+    const int n_chunks = (T + C - 1) / C;
+    if (c >= n_chunks) return;
+    const int Cb = ((T + n_chunks - 1) / n_chunks + kTile - 1) / kTile * kTile;
+    const int t_begin = c * Cb;
+    if (t_begin >= T) return;  // (cannot happen: (n_chunks - 1) * Cb < T)
+    const int t_end = min(T, t_begin + Cb);
+    const int n_tiles = (t_end - t_begin + kTile - 1) / kTile;
+
 
     if (warp == 4) {  // ---------------- producer
         if (lane == 0) {

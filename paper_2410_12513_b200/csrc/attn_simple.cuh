@@ -11,10 +11,10 @@ namespace first {
 // [s*C, min(T,(s+1)*C)) with C = ceil(T/S), T = len[b]+1 (the new token is already written at row len[b]).
 // q: [m][Hq][HD] float32, pre-scaled.  Partials: o_part [m][Hq][S][HD], ml_part [m][Hq][S] = (max, sum).
 template <typename KT, int HD, int G>
-__global__ void __launch_bounds__(128) attn_split_simple(const float* __restrict__ q, const KT* __restrict__ kc,
-                                                         const KT* __restrict__ vc, int64_t cap_total,
+__global__ void __launch_bounds__(128) attn_split_simple(const float* q, const KT* kc,
+                                                         const KT* vc, int64_t cap_total,
                                                          const int64_t* __restrict__ slab_off,
-                                                         const int32_t* __restrict__ len_l,
+                                                         const int32_t* len_l,
                                                          const int32_t* __restrict__ slab_cap,
                                                          const int32_t* __restrict__ idx, int Hq,
                                                          float* __restrict__ o_part, float2* __restrict__ ml_part) {
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* __restrict
 
 // Merge the S partial results of each (row, query head): out[i][hq*HD + d] (float32) and,
 // optionally, its bfloat16 hi/lo split for the tensor-core O-projection.
-__global__ void __launch_bounds__(128) attn_combine(const float* __restrict__ o_part, const float2* __restrict__ ml_part,
+__global__ void __launch_bounds__(128) attn_combine(const float* o_part, const float2* ml_part,
                                                     int S, int HD, float* __restrict__ out,
                                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
     pdl_trigger();

@@ -21,6 +21,9 @@ __device__ __forceinline__ float warp_max(float v) {
 // this one runs, and wait for the previous kernel's results (both are no-ops when the launch
 // carries no programmatic dependency).
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// Everything an earlier kernel of the step produced must be read after this wait.  The "memory" clobber
+// keeps ordinary loads below it, but not loads the compiler may treat as invariant (a const __restrict__
+// kernel parameter): pointers to data produced inside a step therefore carry no __restrict__.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // two packed bfloat16 -> two float32 (a bfloat16 is the upper half of a float32)

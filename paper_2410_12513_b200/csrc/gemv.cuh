@@ -15,7 +15,7 @@ enum GemvEpilogue { kStore = 0, kScatterAdd = 1 };
 //   kScatterAdd: Y[idx[r0+r]*ldy + f]  += dot   (each element owned by one lane: no atomics)
 template <typename WT, int R, int EPI>
 __global__ void __launch_bounds__(256) gemv_rows(const WT* __restrict__ W, int n_out, int K,
-                                                 const float* __restrict__ X, int r0, int rows_valid,
+                                                 const float* X, int r0, int rows_valid,
                                                  float* __restrict__ Y, int64_t ldy, const int32_t* __restrict__ idx) {
     pdl_trigger();
     pdl_wait();

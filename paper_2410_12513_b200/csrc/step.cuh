@@ -61,13 +61,13 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 //             word: x = tokens to attend over (cache length + the new token, at most the slab's
 //             capacity) | batch row << 32;  y = first slab row | (1 << 62 when the new token's key
 //             and value are to be appended).  A full slab raises FIRST_FLAG_KV_FULL.
-__global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x, const int32_t* __restrict__ idx, int D,
+__global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32_t* __restrict__ idx, int D,
                                                      const float* __restrict__ gain, float eps, float* __restrict__ out,
                                                      __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                      float* __restrict__ zero_row, int zero_cols,
                                                      int32_t* __restrict__ len_inc, const int32_t* __restrict__ slab_cap,
                                                      longlong2* __restrict__ rowinfo,
-                                                     const int32_t* __restrict__ len_ro,
+                                                     const int32_t* len_ro,
                                                      const int64_t* __restrict__ slab_off,
                                                      uint32_t* __restrict__ flags) {
     // One pass: the row stays in registers between the sum of squares and the scaling
@@ -142,13 +142,13 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* __restrict__ x
 // rowinfo[i] = (tokens to attend over, first slab row) saves the attention CTAs two dependent loads.
 // A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
-__global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv, const int32_t* __restrict__ idx,
-                                                  int Hq, int Hkv, int hd, const float2* __restrict__ cs,
+__global__ void __launch_bounds__(64) rope_append(const float* qkv, const int32_t* __restrict__ idx,
+                                                  int Hq, int Hkv, int hd, const float2* cs,
                                                   float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
                                                   KT* __restrict__ vc, int64_t cap_total,
                                                   const int64_t* __restrict__ slab_off,
                                                   const int32_t* __restrict__ slab_cap,
-                                                  const int32_t* __restrict__ len_l, uint32_t* __restrict__ flags,
+                                                  const int32_t* len_l, uint32_t* __restrict__ flags,
                                                   longlong2* __restrict__ rowinfo) {
     pdl_trigger();
     pdl_wait();
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(64) rope_append(const float* __restrict__ qkv,
 }
 
 // act[i][f] = silu(gate) * up from gu[i] = [gate(F) | up(F)]; optional bf16 hi/lo split.
-__global__ void __launch_bounds__(256) silu_mul(const float* __restrict__ gu, int m, int F, float* __restrict__ act,
+__global__ void __launch_bounds__(256) silu_mul(const float* gu, int m, int F, float* __restrict__ act,
                                                 __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
     pdl_trigger();
     pdl_wait();
@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(256) silu_mul(const float* __restrict__ gu, in
 
 // End of a step: greedy next token per row (lowest index among equal maxima) and pos += 1.
 // One block of 1024 threads per row; 16-byte loads when the row allows it.
-__global__ void __launch_bounds__(1024) step_end(const float* __restrict__ logits, int V, int32_t* __restrict__ next,
+__global__ void __launch_bounds__(1024) step_end(const float* logits, int V, int32_t* __restrict__ next,
                                                  int32_t* __restrict__ pos) {
     pdl_trigger();
     pdl_wait();
@@ -263,7 +263,7 @@ constexpr int kSampleKMax = 16;
 
 __device__ __forceinline__ bool sample_before(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
 
-__global__ void __launch_bounds__(1024) step_end_sample(const float* __restrict__ logits, int V, int k, float inv_T,
+__global__ void __launch_bounds__(1024) step_end_sample(const float* logits, int V, int k, float inv_T,
                                                         const float* __restrict__ uniforms,
                                                         int32_t* __restrict__ next, int32_t* __restrict__ pos) {
     pdl_trigger();
