@@ -413,7 +413,10 @@ def run_cuda(args, wl, shape, mask, lens):
         traffic = None
     roof = {"bound": "hbm", "kernel": dom, "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "traffic": traffic,
             "traffic_note": "per step, scaled from the 2-layer ncu capture in profiles/ (per launch x launches)" if traffic else None,
-            "ms_per_step": cls_ms[dom], "share_of_kernel_time": cls_ms[dom] / tot_cls}
+            "ms_per_step": cls_ms[dom], "share_of_kernel_time": cls_ms[dom] / tot_cls,
+            "timing": "CUDA event pair around every launch of the class, summed over a profiled pass of the timed steps; "
+                      "the events serialise the launches, so the overlap between neighbouring kernels that a normal step "
+                      "has (weight tiles requested before the dependency wait) is absent: a lower bound on the in-step rate"}
     if dom in alg:
         roof["achieved"] = alg[dom] / cls_ms[dom] / 1e6
         roof["frac"] = roof["achieved"] / peak
