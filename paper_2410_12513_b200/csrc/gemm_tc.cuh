@@ -150,12 +150,36 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
     const int kb0 = (int)((int64_t)p.kblocks * split / p.ksplit), kb1 = (int)((int64_t)p.kblocks * (split + 1) / p.ksplit);
     const int nkb = kb1 - kb0;
 
+    // Thread 0 is the TMA producer.  It sets the barriers up and at once asks for the first weight tiles:
+    // they depend neither on the previous kernel nor on the rest of this CTA's set-up (TMEM allocation, the
+    // CTA-wide barrier), so HBM is already streaming while those happen.
+    uint64_t pol_stream = 0;
+    const uint32_t tx = (EPI == kEpiSwiglu && p.mt == 1)
+                            ? (uint32_t)(stage_bytes - a_bytes + 2 * p.pair_rows * 128)  // two boxes of R rows
+                            : (uint32_t)stage_bytes;
+    auto load_a = [&](uint32_t sa, uint32_t bar, int kc) {
+        if (EPI == kEpiSwiglu) {
+            // gate rows, then the matching up rows: R+R (mt = 1, R = pair_rows <= 64) or 128+128 (mt = 2)
+            const int rows = p.mt == 1 ? p.pair_rows : 128;
+            const CUtensorMap* tm = p.mt == 1 ? &tmA : &tmA2;
+            tma_load_2d_hint(sa, tm, bar, kc, tile * rows, pol_stream);
+            tma_load_2d_hint(sa + rows * 128, tm, bar, kc, p.n_out + tile * rows, pol_stream);
+        } else {
+            for (int a = 0; a < p.mt; ++a)
+                tma_load_2d_hint(sa + a * kABytes, &tmA, bar, kc, (tile * p.mt + a) * kBlockM, pol_stream);
+        }
+    };
+    const int npre = min(p.stages, nkb);
     if (threadIdx.x == 0) {
         abort_s = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(tmem_full_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+        for (int i = 0; i < npre; ++i) {
+            mbar_expect_tx(full_bar(i), tx);
+            load_a(base + (uint32_t)i * stage_bytes, full_bar(i), (kb0 + i) * kBlockK);
+        }
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBh) : "memory");
         if (p.use_lo) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBl) : "memory");
     }
@@ -171,30 +195,8 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
 
     if (warp == 0) {
         if (lane == 0) {
-            uint64_t pol_stream;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            const uint32_t tx = (EPI == kEpiSwiglu && p.mt == 1)
-                                    ? (uint32_t)(stage_bytes - a_bytes + 2 * p.pair_rows * 128)  // two boxes of R rows
-                                    : (uint32_t)stage_bytes;
-            auto load_a = [&](uint32_t sa, uint32_t bar, int kc) {
-                if (EPI == kEpiSwiglu) {
-                    // gate rows, then the matching up rows: R+R (mt = 1, R = pair_rows <= 64) or 128+128 (mt = 2)
-                    const int rows = p.mt == 1 ? p.pair_rows : 128;
-                    const CUtensorMap* tm = p.mt == 1 ? &tmA : &tmA2;
-                    tma_load_2d_hint(sa, tm, bar, kc, tile * rows, pol_stream);
-                    tma_load_2d_hint(sa + rows * 128, tm, bar, kc, p.n_out + tile * rows, pol_stream);
-                } else {
-                    for (int a = 0; a < p.mt; ++a)
-                        tma_load_2d_hint(sa + a * kABytes, &tmA, bar, kc, (tile * p.mt + a) * kBlockM, pol_stream);
-                }
-            };
-            // Weights do not depend on the previous kernel: fill the ring with weight tiles first,
-            // then wait for the previous kernel and add the activation tiles to the same stages.
-            const int npre = min(p.stages, nkb);
-            for (int i = 0; i < npre; ++i) {
-                mbar_expect_tx(full_bar(i), tx);
-                load_a(base + (uint32_t)i * stage_bytes, full_bar(i), (kb0 + i) * kBlockK);
-            }
+            // The ring already holds requests for the first weight tiles (set-up above): wait for the
+            // previous kernel and add the activation tiles to the same stages.
             pdl_wait();
             for (int i = 0; i < npre; ++i) {
                 const uint32_t sa = base + (uint32_t)i * stage_bytes;
