@@ -137,7 +137,7 @@ int first_destroy(first_ctx *ctx);
  *   router_w      dev float32 [d_model];  router_b  dev float32 [1] or NULL
  *   mask          dev uint8 [B][n_layers] (only column `layer` is written)
  *   scores        dev float32 [B][n_layers] or NULL
- * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_CUDA. */
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_UNSUPPORTED (d_model > 12288), FIRST_E_CUDA. */
 int first_prefill_route(first_ctx *ctx, int32_t layer, const void *hidden, int32_t hidden_dtype,
                         const int32_t *cu_seqlens, int32_t B, int64_t total_tokens, const float *router_w,
                         const float *router_b, float tau, int32_t mode, uint8_t *mask, float *scores,

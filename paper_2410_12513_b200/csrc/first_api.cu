@@ -687,6 +687,7 @@ int first_prefill_route(first_ctx* c, int32_t layer, const void* hidden, int32_t
     if (total_tokens > c->tok_cap || total_tokens > 0x7fffffffLL) return FIRST_E_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int D = c->d.d_model;
+    if (D > 12288) return FIRST_E_UNSUPPORTED;  // the router vector is staged in 48 KB of shared memory
     const int64_t want = (total_tokens + 7) / 8;
     const int blocks = (int)std::min<int64_t>(want, (int64_t)c->n_sm * 8);
     const size_t smem = (size_t)D * sizeof(float);

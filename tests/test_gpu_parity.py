@@ -262,6 +262,40 @@ def test_full_slab_sets_flag_and_leaves_cache():
     assert gkv.len.cpu().numpy()[:, 1].tolist() == [5] * shape.n_layers
 
 
+def test_full_slab_on_the_tuned_attention_path():
+    """bfloat16 cache, head_dim 128: the attention kernel itself appends the new key/value; a full slab must be
+    left alone (flag raised, length kept) while the other sequence appends as usual."""
+    import torch
+    shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
+    w = fi.make_weights(shape, 2, True)
+    okv, gkv = synthetic_caches(shape, [70, 70], [70, 72], 1, True)
+    ctx = _ctx(shape, True, 2, 80, w)
+    ctx.set_mask(torch.ones((2, shape.n_layers), dtype=torch.uint8, device="cuda"))
+    full_before = [gkv.rows_host(l, 0) for l in range(shape.n_layers)]
+    logits = torch.empty((2, shape.vocab), dtype=torch.float32, device="cuda")
+    toks = fi.tokens(shape, 2, 5, "t")
+    ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits)
+    assert ctx.device_flags() == 1  # FIRST_FLAG_KV_FULL
+    for l in range(shape.n_layers):
+        k1, v1 = gkv.rows_host(l, 0)
+        assert np.array_equal(k1, full_before[l][0]) and np.array_equal(v1, full_before[l][1])
+    assert gkv.len.cpu().numpy()[:, 0].tolist() == [70] * shape.n_layers
+    assert gkv.len.cpu().numpy()[:, 1].tolist() == [71] * shape.n_layers
+    # the sequence with room is unaffected by its neighbour: same logits as when it runs alone
+    om = oracle_model(shape, w)
+    okv1, _ = synthetic_caches(shape, [70, 70], [70, 72], 1, True, with_gpu=False)
+    solo = oracle.OracleKV(oracle.Shape(**shape.asdict()), [72])
+    for l in range(shape.n_layers):
+        ks, vs = okv1.rows(l, 1)
+        kd, vd = solo.rows(l, 0)
+        kd[:], vd[:] = ks, vs
+    solo.len[:] = 70
+    solo.pos[:] = 70
+    ref = oracle.decode_step(om, toks[1:2], np.ones((1, shape.n_layers), np.uint8), solo)
+    err, _ = logits_check(logits[1:2].cpu().numpy(), ref)
+    assert err.max() <= 2e-2
+
+
 def test_bad_token_sets_flag():
     import torch
     shape = fi.TINY
