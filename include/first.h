@@ -107,7 +107,15 @@ typedef struct {
     const int32_t *slab_cap; /* dev [B] */
     int32_t *len;            /* dev [L][B], updated by first_decode_step */
     int32_t *pos;            /* dev [B],    updated by first_decode_step */
-    int64_t cap_total;       /* token rows per head in each layer tensor */
+    int64_t cap_total;       /* token rows per head in each layer tensor (per_layer = 0) */
+    /* Per-layer slab tables.  A sequence that skips layer l needs no cache there during decode
+     * ("Inference for FiRST", item 2), so once the masks are known a caller can keep, per layer,
+     * slabs only for the sequences that keep it and hand the memory of the others back.  With
+     * per_layer = 1: slab_off is dev [L][B], slab_cap dev [L][B] (0 for a skipped (l,b); its
+     * slab_off is ignored), layer l's tensors are [Hkv][cap_total_l[l]][hd], cap_total is unused.
+     * The heights are baked into recorded step graphs: call first_set_mask after changing them. */
+    int32_t per_layer;             /* 0 (tables shared by all layers) or 1 */
+    const int64_t *cap_total_l;    /* host [L], per_layer = 1 only */
 } first_kv_cache;
 
 /* Create a context for one model on the current device: validates the description,

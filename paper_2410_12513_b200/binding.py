@@ -39,7 +39,8 @@ class Weights(C.Structure):
 
 class KVCacheC(C.Structure):
     _fields_ = [("k", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)), ("slab_off", C.c_void_p),
-                ("slab_cap", C.c_void_p), ("len", C.c_void_p), ("pos", C.c_void_p), ("cap_total", C.c_int64)]
+                ("slab_cap", C.c_void_p), ("len", C.c_void_p), ("pos", C.c_void_p), ("cap_total", C.c_int64),
+                ("per_layer", C.c_int32), ("cap_total_l", C.POINTER(C.c_int64))]
 
 
 def library_path() -> Path:
@@ -121,16 +122,24 @@ class KVCache:
 
     k, v: lists (one per layer) of CUDA tensors [Hkv][cap_total][hd] (None allowed for
     layers no sequence keeps); slab_off int64 [B]; slab_cap int32 [B]; len int32 [L][B];
-    pos int32 [B]."""
+    pos int32 [B].  With two-dimensional slab_off / slab_cap ([L][B]) the tables are per
+    layer and every layer's tensors may have their own height (a layer then holds slabs
+    only for the sequences that keep it)."""
 
     def __init__(self, k, v, slab_off, slab_cap, len_, pos):
         self.k, self.v, self.slab_off, self.slab_cap, self.len, self.pos = k, v, slab_off, slab_cap, len_, pos
         first = next(t for t in k if t is not None)
         self._ka = _ptr_array(k, first.dtype, "kv.k")
         self._va = _ptr_array(v, first.dtype, "kv.v")
+        per_layer = slab_off.dim() == 2
+        if per_layer != (slab_cap.dim() == 2):
+            raise ValueError("slab_off and slab_cap must both be [B] or both be [L][B]")
+        self._heights = (C.c_int64 * len(k))(*[0 if t is None else int(t.shape[1]) for t in k])
         self.c = KVCacheC(C.cast(self._ka, C.POINTER(C.c_void_p)), C.cast(self._va, C.POINTER(C.c_void_p)),
                           _dev(slab_off, torch.int64, "slab_off"), _dev(slab_cap, torch.int32, "slab_cap"),
-                          _dev(len_, torch.int32, "len"), _dev(pos, torch.int32, "pos"), int(first.shape[1]))
+                          _dev(len_, torch.int32, "len"), _dev(pos, torch.int32, "pos"),
+                          0 if per_layer else int(first.shape[1]), int(per_layer),
+                          C.cast(self._heights, C.POINTER(C.c_int64)))
 
 
 def first_create(shape, dtype, max_batch, max_tokens_per_seq, weights):

@@ -331,9 +331,21 @@ int launch_gemv(first_ctx* c, cudaStream_t st, const void* W, int n_out, int K, 
     return FIRST_OK;
 }
 
+// One layer's view of the cache tables: shared by all layers, or (first_kv_cache::per_layer) this layer's
+// rows of the [L][B] tables and its own tensor height.
+struct LayerKv {
+    const int64_t* slab_off;
+    const int32_t* slab_cap;
+    int64_t cap_total;
+};
+LayerKv layer_kv(const first_kv_cache* kv, int l, int B) {
+    if (!kv->per_layer) return {kv->slab_off, kv->slab_cap, kv->cap_total};
+    return {kv->slab_off + (size_t)l * B, kv->slab_cap + (size_t)l * B, kv->cap_total_l[l]};
+}
+
 template <typename KT, int HD>
 int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* kc, const KT* vc,
-                         const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx) {
+                         const LayerKv* kv, const int32_t* len_l, const int32_t* idx) {
     dim3 grid(S, c->d.n_kv_heads, m);
 #define FIRST_ATTN_CASE(G)                                                                                  \
     case G:                                                                                                 \
@@ -354,7 +366,7 @@ int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* 
 
 template <typename KT>
 int launch_attn_simple(first_ctx* c, cudaStream_t st, int S, int m, const void* kc, const void* vc,
-                       const first_kv_cache* kv, const int32_t* len_l, const int32_t* idx) {
+                       const LayerKv* kv, const int32_t* len_l, const int32_t* idx) {
     const KT *k = static_cast<const KT*>(kc), *v = static_cast<const KT*>(vc);
     switch (c->d.head_dim) {
         case 32: return launch_attn_simple_g<KT, 32>(c, st, S, m, k, v, kv, len_l, idx);
@@ -379,7 +391,7 @@ int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorM
 
 template <int HD, int G>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
-                       const first_kv_cache* kv, const void* kc, const void* vc, int C, float* out,
+                       const LayerKv* kv, const void* kc, const void* vc, int C, float* out,
                        __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     attn::RopeFuse rf{};
@@ -413,7 +425,7 @@ int attn_mma_setup(first_ctx* c) {
 }
 
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
-int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const first_kv_cache* kv,
+int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const LayerKv* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
                     __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
     const first_model_desc& d = c->d;
@@ -493,6 +505,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool t = tc_for(m);
         const int32_t* idx = c->idx + (size_t)l * B;
         int32_t* len_l = kv->len + (size_t)l * B;
+        const LayerKv lkv = layer_kv(kv, l, B);
         float* f32 = t ? nullptr : c->xn;
         __nv_bfloat16 *xh = t ? c->xh : nullptr, *xl = t ? c->xl : nullptr;
         // split-K projections reduce into float32 accumulators that the preceding norm kernel clears
@@ -502,8 +515,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, static_cast<int32_t*>(nullptr),
-                           fuse_rope ? kv->slab_cap : nullptr, fuse_rope ? c->rowinfo : nullptr,
-                           fuse_rope ? static_cast<const int32_t*>(len_l) : nullptr, fuse_rope ? kv->slab_off : nullptr,
+                           fuse_rope ? lkv.slab_cap : nullptr, fuse_rope ? c->rowinfo : nullptr,
+                           fuse_rope ? static_cast<const int32_t*>(len_l) : nullptr, fuse_rope ? lkv.slab_off : nullptr,
                            c->flags)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
@@ -514,15 +527,15 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         if (!fuse_rope &&
             (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
                            0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
-                           static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), kv->cap_total, kv->slab_off,
-                           kv->slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr)))
+                           static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
+                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr)))
             return rc;
         if (mma_attn) {
-            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], kv, len_l, idx, t ? nullptr : c->att, xh, xl,
+            if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], &lkv, len_l, idx, t ? nullptr : c->att, xh, xl,
                                       fuse_rope, qscale)))
                 return rc;
         } else {
-            if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], kv, len_l, idx))) return rc;
+            if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], &lkv, len_l, idx))) return rc;
             if ((rc = launch_k(c, st, kClsAttnCombine, attn_combine, dim3(m * d.n_q_heads), dim3(128), 0, c->o_part,
                                c->ml_part, S, hd, t ? nullptr : c->att, xh, xl)))
                 return rc;
@@ -532,7 +545,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             return rc;
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->ffn_norm[l],
-                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, kv->slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
+                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, lkv.slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
@@ -740,10 +753,13 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
                       int32_t* next_tokens, float* layer_inputs, void* stream) {
     if (!c || !tokens || !kv) return FIRST_E_ARG;
     if (!c->has_mask) return FIRST_E_STATE;
-    if (!kv->k || !kv->v || !kv->slab_off || !kv->slab_cap || !kv->len || !kv->pos || kv->cap_total <= 0)
-        return FIRST_E_ARG;
-    for (int l = 0; l < c->d.n_layers; ++l)
-        if (c->cnt_h[l] > 0 && (!kv->k[l] || !kv->v[l])) return FIRST_E_ARG;
+    if (!kv->k || !kv->v || !kv->slab_off || !kv->slab_cap || !kv->len || !kv->pos) return FIRST_E_ARG;
+    if (kv->per_layer ? !kv->cap_total_l : kv->cap_total <= 0) return FIRST_E_ARG;
+    for (int l = 0; l < c->d.n_layers; ++l) {
+        if (c->cnt_h[l] == 0) continue;
+        if (!kv->k[l] || !kv->v[l]) return FIRST_E_ARG;
+        if (kv->per_layer && kv->cap_total_l[l] <= 0) return FIRST_E_ARG;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto run = [&](cudaStream_t s) {
         if (c->d.dtype == FIRST_DTYPE_BF16)
@@ -764,6 +780,10 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     key.push_back(tokens); key.push_back(logits); key.push_back(next_tokens); key.push_back(layer_inputs);
     key.push_back(kv->slab_off); key.push_back(kv->slab_cap); key.push_back(kv->len); key.push_back(kv->pos);
     key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->cap_total)));
+    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->per_layer)));
+    if (kv->per_layer)
+        for (int l = 0; l < c->d.n_layers; ++l)
+            key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->cap_total_l[l])));
     key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->plan_version)));
     for (int l = 0; l < c->d.n_layers; ++l) { key.push_back(kv->k[l]); key.push_back(kv->v[l]); }
     first_ctx::StepGraph* g = nullptr;

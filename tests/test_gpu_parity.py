@@ -518,3 +518,63 @@ def test_decode_step_samples_when_asked():
                 assert tok[b] == got[b].argmax()
         toks = oracle.argmax(ref)
     assert ctx.device_flags() == 0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_per_layer_slab_tables(bf16):
+    """Once the masks are fixed a layer only needs slabs for the sequences that keep it ("Inference for
+    FiRST", item 2).  The same decode, run from caches that hold exactly those slabs (per-layer tables,
+    per-layer tensor heights), gives the same logits as from full caches (bit for bit on the float32 path),
+    and the oracle's."""
+    import torch
+    from paper_2410_12513_b200 import KVCache
+    shape = fi.ModelShape(3, 256, 8, 2, 128, 512, 1000, 500000.0) if bf16 else fi.TINY
+    seed, B, steps = 51, 6, 3
+    L = shape.n_layers
+    w = fi.make_weights(shape, seed, bf16)
+    om = oracle_model(shape, w)
+    lens = fi.prompt_lengths(B, 1, 150, seed)
+    caps = [int(n) + steps + (b % 2) for b, n in enumerate(lens)]
+    mask = fi.mask_bernoulli(B, L, 0.6, seed)
+    mask[:, 1] = 0  # a layer nobody keeps: no tensors at all for it
+    okv, gkv = synthetic_caches(shape, lens, caps, seed, bf16)
+    # per-layer caches: only the kept sequences' slabs, packed
+    k2, v2 = [None] * L, [None] * L
+    off2 = np.zeros((L, B), np.int64)
+    cap2 = np.zeros((L, B), np.int32)
+    for l in range(L):
+        kept = [b for b in range(B) if mask[b, l]]
+        if not kept:
+            continue
+        cap2[l, kept] = [caps[b] for b in kept]
+        off2[l, kept] = np.concatenate([[0], np.cumsum([caps[b] for b in kept])[:-1]])
+        height = int(cap2[l].sum())
+        k2[l] = torch.zeros((shape.n_kv_heads, height, shape.head_dim), dtype=gkv.k[l].dtype, device="cuda")
+        v2[l] = torch.zeros_like(k2[l])
+        for b in kept:
+            o, o2, cp = int(gkv.off[b]), int(off2[l, b]), caps[b]
+            k2[l][:, o2:o2 + cp] = gkv.k[l][:, o:o + cp]
+            v2[l][:, o2:o2 + cp] = gkv.v[l][:, o:o + cp]
+    full_rows = L * sum(caps)
+    kept_rows = int(cap2.sum())
+    assert kept_rows == sum(caps[b] for b in range(B) for l in range(L) if mask[b, l]) and kept_rows < 0.75 * full_rows
+    kv2 = KVCache(k2, v2, torch.from_numpy(off2).cuda(), torch.from_numpy(cap2).cuda(), gkv.len.clone(), gkv.pos.clone())
+    ctx = _ctx(shape, bf16, B, max(caps), w)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    la = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda")
+    lb = torch.empty_like(la)
+    toks = fi.tokens(shape, B, seed, "first")
+    for _ in range(steps):
+        ref = oracle.decode_step(om, toks, mask, okv)
+        td = torch.from_numpy(toks).cuda()
+        ctx.decode_step(td, gkv.c, la)
+        ctx.decode_step(td, kv2, lb)
+        assert ctx.device_flags() == 0
+        if bf16:  # the tensor-core projections reduce K ranges with float atomics: run-to-run order differs
+            assert logits_check(lb.cpu().numpy(), la.cpu().numpy())[0].max() <= 1e-4
+        else:
+            assert torch.equal(la, lb)
+        err, _ = logits_check(lb.cpu().numpy(), ref)
+        assert err.max() <= (2e-2 if bf16 else 1e-4)
+        toks = oracle.argmax(ref)
+    assert torch.equal(kv2.len, gkv.len) and torch.equal(kv2.pos, gkv.pos)
