@@ -164,8 +164,9 @@ def test_zz_argmax_agreement_over_all_scale_cases():
     """Aggregate over every (step, sequence) pair checked above."""
     import json, os
     print(json.dumps(_tally))
-    if os.path.isdir("gpurun_out"):
-        with open("gpurun_out/scale_parity.json", "w") as f:
+    report = os.environ.get("FIRST_PARITY_REPORT")  # optional: a file to leave the tally in
+    if report:
+        with open(report, "w") as f:
             json.dump(_tally, f)
     if _tally["n"] < 100:
         pytest.skip("run together with the scale cases")
