@@ -97,12 +97,12 @@ struct first_ctx {
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
-    int tc_mt2_min_rows = 1 << 30;
+    int tc_mt2_min_rows = 1 << 30;  // from this many active rows on, a projection CTA takes two weight tiles
+    int tc_ksplit_cap = 1;          // bound the number of K ranges by the reduction traffic they add
     // sampling of the next token (greedy while sample_k <= 1)
     int sample_k = 0;
     float sample_inv_T = 1.f;
     const float* sample_u = nullptr;
-    int tc_ksplit_cap = 1;  // from this many active rows on, a projection CTA takes two weight tiles
 };
 
 constexpr int kSimpleSplitsMax = 16;
