@@ -578,3 +578,42 @@ def test_per_layer_slab_tables(bf16):
         assert err.max() <= (2e-2 if bf16 else 1e-4)
         toks = oracle.argmax(ref)
     assert torch.equal(kv2.len, gkv.len) and torch.equal(kv2.pos, gkv.pos)
+
+
+def test_documented_error_statuses():
+    """The statuses the header promises: unsupported shapes at create, call order, capacity, sampling limits."""
+    import dataclasses
+    import torch
+    from paper_2410_12513_b200 import FirstError
+    w = fi.make_weights(fi.TINY, 3, False)
+    gw = gpu_weights(w)
+    from paper_2410_12513_b200 import FirstContext
+
+    def create_status(shape):
+        try:
+            FirstContext(shape, F32, 2, 16, gw)
+        except FirstError as e:
+            return e.status
+        return 0
+
+    assert create_status(dataclasses.replace(fi.TINY, n_q_heads=5, n_kv_heads=1, head_dim=64)) == -3   # 5 query heads per KV head
+    assert create_status(dataclasses.replace(fi.TINY, head_dim=48)) in (-2, -3)                        # head_dim not 32/64/128
+    assert create_status(dataclasses.replace(fi.TINY, n_q_heads=4, n_kv_heads=3)) == -2                # heads do not divide
+    ctx = _ctx(fi.TINY, False, 2, 16, w)
+    _, gkv = synthetic_caches(fi.TINY, [3, 3], [8, 8], 1, False)
+    toks = torch.zeros(2, dtype=torch.int32, device="cuda")
+    with pytest.raises(FirstError) as e:   # decode before any mask
+        ctx.decode_step(toks, gkv.c)
+    assert e.value.status == -7
+    with pytest.raises(FirstError) as e:   # batch beyond max_batch
+        ctx.set_mask(torch.ones((3, fi.TINY.n_layers), dtype=torch.uint8, device="cuda"))
+    assert e.value.status == -4
+    with pytest.raises(FirstError) as e:   # top_k beyond the device limit
+        ctx.set_sampling(17, 0.8, torch.zeros(2, device="cuda"))
+    assert e.value.status == -3
+    with pytest.raises(FirstError) as e:   # sampling without draws
+        ctx.set_sampling(10, 0.8, None)
+    assert e.value.status == -1
+    ctx.set_mask(torch.ones((2, fi.TINY.n_layers), dtype=torch.uint8, device="cuda"))
+    ctx.decode_step(toks, gkv.c)           # and the context still works afterwards
+    assert ctx.device_flags() == 0
