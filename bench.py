@@ -330,10 +330,11 @@ def run_cuda(args, wl, shape, mask, lens):
     repeat_ms, _ = timed(mask_t)  # the routed run once more, after the dense one (order effects show here)
     repeat_ms /= K
 
-    sweep = None
-    if args.sweep:
-        sweep = []
-        for frac in (0.0, 0.1, 0.2, 0.3, 0.4, 0.5):
+    # Step latency against the skip rate, on this workload's batch and caches: always a short version (three
+    # rates, both mask structures), the six rates of the sweep config with --sweep.
+    sweep = []
+    if True:
+        for frac in ((0.0, 0.1, 0.2, 0.3, 0.4, 0.5) if args.sweep else (0.0, 0.25, 0.5)):
             row = {"skip": frac}
             for kind in ("aligned", "independent"):
                 mk = fi.mask_aligned(B, L, frac) if kind == "aligned" else fi.mask_independent(B, L, frac, 3000 + rank)
@@ -468,7 +469,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
     ap.add_argument("--sweep", action="store_true",
-                    help="also time skip fractions 0..50 %% (aligned and independent masks) on this workload")
+                    help="time six skip fractions 0..50 %% (aligned and independent masks) on this workload instead of three")
     ap.add_argument("--quick", action="store_true",
                     help="only the main timed loop (for profiler captures): no dense/e2e/per-kernel legs")
     args = ap.parse_args()
