@@ -617,3 +617,28 @@ def test_documented_error_statuses():
     ctx.set_mask(torch.ones((2, fi.TINY.n_layers), dtype=torch.uint8, device="cuda"))
     ctx.decode_step(toks, gkv.c)           # and the context still works afterwards
     assert ctx.device_flags() == 0
+
+
+def test_next_tokens_without_a_logits_buffer():
+    """next_tokens alone (the library keeps the logits to itself) gives the same tokens as asking for both,
+    greedy and sampled."""
+    import torch
+    shape, seed, B = fi.TINY, 61, 4
+    w = fi.make_weights(shape, seed, False)
+    lens = [5, 9, 3, 12]
+    ctx = _ctx(shape, False, B, 24, w)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.7, seed)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = torch.from_numpy(fi.tokens(shape, B, seed, "t")).cuda()
+    u = torch.tensor([0.1, 0.5, 0.7, 0.95], dtype=torch.float32, device="cuda")
+    for sampled in (False, True):
+        ctx.set_sampling(10 if sampled else 0, 0.8 if sampled else 0.0, u if sampled else None)
+        out = []
+        for with_logits in (True, False):
+            _, gkv = synthetic_caches(shape, lens, [16] * B, seed, False)
+            nxt = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+            logits = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda") if with_logits else None
+            ctx.decode_step(toks, gkv.c, logits, nxt)
+            assert ctx.device_flags() == 0
+            out.append(nxt.cpu().numpy())
+        assert (out[0] >= 0).all() and np.array_equal(out[0], out[1])
