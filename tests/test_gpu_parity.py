@@ -166,9 +166,10 @@ def test_decode_bf16_gqa_ragged(shape):
     assert agrees.mean() >= 0.9  # tiny vocab-independent sanity; the aggregate bar is checked at scale
 
 
-@pytest.mark.parametrize("B", [70, 200])
-def test_decode_bf16_many_rows_two_tile_projection(B):
-    """Enough active rows that a projection CTA takes two weight tiles per activation tile."""
+@pytest.mark.parametrize("B", [70, 200, 300])
+def test_decode_bf16_many_rows(B):
+    """Many active rows: wide activation tiles (one projection CTA per SM), and with 300 rows more than one
+    256-row projection launch per matrix."""
     shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
     lens = fi.prompt_lengths(B, 1, 90, 13)
     mask = fi.mask_bernoulli(B, shape.n_layers, 0.85, 14)
