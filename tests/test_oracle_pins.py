@@ -373,3 +373,20 @@ def test_sampling_rejects_bad_arguments():
     for k, T, u in ((0, 1.0, 0.5), (5, 1.0, 0.5), (2, -1.0, 0.5), (2, 1.0, 1.0), (2, 1.0, -0.1)):
         with pytest.raises(RuntimeError):
             oracle.sample_topk(z, k, T, u)
+
+
+def _sampling_rows():
+    rows = []
+    for line in (GOLDEN / "sampling_hand_examples.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        name, logits, k, T, cands, p0 = [c.strip() for c in line.split("|")]
+        rows.append((name, [float(x) for x in logits.split()], int(k), float(T), [int(x) for x in cands.split()], float(p0)))
+    return rows
+
+
+@pytest.mark.parametrize("name,logits,k,T,cands,p0", _sampling_rows())
+def test_sampling_hand_examples(name, logits, k, T, cands, p0):
+    _, cand, prob = oracle.sample_topk(np.array(logits, np.float32), k, T, 0.0)
+    assert list(cand) == cands
+    assert abs(prob[0] - p0) < 1e-6 and abs(prob.sum() - 1.0) < 1e-12
