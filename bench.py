@@ -142,48 +142,62 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- oracle arm
-def oracle_sample(shape, mask, lens, seed, rows=4, layers=2):
-    """Time the host oracle on a bounded sample of the workload: `rows` sequences of the batch
-    (their real cache lengths, stand-in cache contents), `layers` decoder layers of the same
-    width, plus final norm + lm_head; extrapolate to the whole step by the mask's kept
+class OracleSample:
+    """A bounded sample of the workload for the host oracle: `rows` sequences of the batch (their real cache
+    lengths, stand-in cache contents), `layers` decoder layers of the same width, plus final norm + lm_head.
+    step() times one decode step of the sample and extrapolates to the whole step by the mask's kept
     (row, layer) count."""
-    sys.path.insert(0, str(ROOT / "tests"))
-    import oracle
-    from harness import oracle_model, synthetic_caches
-    B, L = mask.shape
-    rows = min(rows, B)
-    sub = fi.ModelShape(layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn_dim,
-                        shape.vocab, shape.rope_base, shape.rms_eps)
-    w = fi.make_weights(sub, seed, True)
-    om = oracle_model(sub, w)
-    sel = np.linspace(0, B - 1, rows).astype(int)
-    l_sel = [int(lens[b]) for b in sel]
-    okv, _ = synthetic_caches(sub, l_sel, [n + 2 for n in l_sel], seed, True, with_gpu=False)
-    toks = fi.tokens(sub, rows, seed, "oracle_tokens")
-    t0 = time.perf_counter()
-    oracle.decode_step(om, toks, np.zeros((rows, layers), np.uint8), okv)
-    t_head = (time.perf_counter() - t0) / rows
-    t0 = time.perf_counter()
-    oracle.decode_step(om, toks, np.ones((rows, layers), np.uint8), okv)
-    t_all = time.perf_counter() - t0
-    t_layer = max(t_all - t_head * rows, 0.0) / (rows * layers)
-    kept = int(mask.sum())
-    step_s = kept * t_layer + B * t_head
-    cores = len(os.sched_getaffinity(0))
-    return dict(value=B / step_s, unit=UNIT, cores=cores, kind="oracle",
-                sample=f"{rows} of {B} sequences x {layers} of {L} layers + lm_head, 1 step, bf16-valued weights; "
-                       f"{t_layer * 1e3:.1f} ms per (sequence, kept layer), {t_head * 1e3:.1f} ms per sequence for "
-                       f"norm+lm_head; extrapolated to {kept} kept (sequence, layer) pairs",
-                ms_per_step=step_s * 1e3)
+
+    def __init__(self, shape, mask, lens, seed, rows=4, layers=2):
+        sys.path.insert(0, str(ROOT / "tests"))
+        import oracle
+        from harness import oracle_model, synthetic_caches
+        self.oracle = oracle
+        self.B, self.L = mask.shape
+        self.rows, self.layers = min(rows, self.B), layers
+        self.kept = int(mask.sum())
+        sub = fi.ModelShape(layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn_dim,
+                            shape.vocab, shape.rope_base, shape.rms_eps)
+        self.om = oracle_model(sub, fi.make_weights(sub, seed, True))
+        sel = np.linspace(0, self.B - 1, self.rows).astype(int)
+        l_sel = [int(lens[b]) for b in sel]
+        self.caps = [n + 2 for n in l_sel]
+        self.okv, _ = synthetic_caches(sub, l_sel, self.caps, seed, True, with_gpu=False)
+        self.len0, self.pos0 = self.okv.len.copy(), self.okv.pos.copy()
+        self.toks = fi.tokens(sub, self.rows, seed, "oracle_tokens")
+
+    def step(self):
+        rows, layers, oracle = self.rows, self.layers, self.oracle
+        self.okv.len[:], self.okv.pos[:] = self.len0, self.pos0  # every timed step sees the same cache lengths
+        t0 = time.perf_counter()
+        oracle.decode_step(self.om, self.toks, np.zeros((rows, layers), np.uint8), self.okv)
+        t_head = (time.perf_counter() - t0) / rows
+        self.okv.pos[:] = self.pos0
+        t0 = time.perf_counter()
+        oracle.decode_step(self.om, self.toks, np.ones((rows, layers), np.uint8), self.okv)
+        t_all = time.perf_counter() - t0
+        t_layer = max(t_all - t_head * rows, 0.0) / (rows * layers)
+        step_s = self.kept * t_layer + self.B * t_head
+        cores = len(os.sched_getaffinity(0))
+        return dict(value=self.B / step_s, unit=UNIT, cores=cores, kind="oracle",
+                    sample=f"{rows} of {self.B} sequences x {layers} of {self.L} layers + lm_head, 1 step, bf16-valued "
+                           f"weights; {t_layer * 1e3:.1f} ms per (sequence, kept layer), {t_head * 1e3:.1f} ms per "
+                           f"sequence for norm+lm_head; extrapolated to {self.kept} kept (sequence, layer) pairs",
+                    ms_per_step=step_s * 1e3)
+
+
+def oracle_sample(shape, mask, lens, seed, rows=4, layers=2):
+    return OracleSample(shape, mask, lens, seed, rows, layers).step()
 
 
 def run_reference(args, wl, shape, mask, lens):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    sample = OracleSample(shape, mask, lens, 100, rows=min(mask.shape[0], 8), layers=2)  # built once, stepped K times
     vals = []
     for i in range(args.warmup + args.steps):
-        r = oracle_sample(shape, mask, lens, 100 + i, rows=2, layers=1)
+        r = sample.step()
         if i >= args.warmup:
             vals.append(r)
     ms = float(np.mean([v["ms_per_step"] for v in vals]))
@@ -194,7 +208,10 @@ def run_reference(args, wl, shape, mask, lens):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-           "config": {"workload": args.workload, "note": "host oracle on a bounded sample, extrapolated"},
+           "config": {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": int(mask.shape[0]),
+                      "prompt_lengths": [int(lens.min()), int(lens.max())], "mask": list(wl["mask"]),
+                      "skip_fraction": float(1 - mask.mean()),
+                      "note": "host oracle on a bounded sample of this workload, extrapolated"},
            "cpu_baseline": cb,
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
