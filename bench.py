@@ -496,8 +496,6 @@ def main():
         wl["mask"] = tuple([parts[0]] + [float(x) for x in parts[1:]])
     if args.steps is None:
         args.steps = 64 if args.impl == "cuda" else 2
-    if args.impl == "reference" and args.warmup > 1:
-        args.warmup = 1
     if args.impl == "cuda" and not args.quick:
         args.warmup = max(args.warmup, 3)
     shape = SHAPES[wl["shape"]]
