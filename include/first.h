@@ -279,7 +279,8 @@ const char *first_kernel_class_name(int32_t k);
  *                    active rows, the hi half alone above (default: always both halves; the hi
  *                    half alone is bfloat16-activation accuracy and misses the parity bar)
  *   "tc_mt2_min_rows" from this many active rows on a projection CTA takes two weight tiles per
- *                    activation tile (default: never)
+ *                    activation tile (default: when the activation tiles are so wide that only one
+ *                    single-tile CTA would fit per SM, i.e. from 96 rows)
  *   "tc_ksplit_cap"  0 = do not bound the number of K ranges by the reduction traffic
  *   "tc_smem_kb"     shared-memory budget per projection CTA when two CTAs per SM are wanted (110)
  *   "fuse_rope"      0 = a separate kernel rotates q/k and appends the new key/value before attention.

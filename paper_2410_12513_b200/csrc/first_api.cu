@@ -97,7 +97,7 @@ struct first_ctx {
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
-    int tc_mt2_min_rows = 1 << 30;  // from this many active rows on, a projection CTA takes two weight tiles
+    int tc_mt2_min_rows = -1;  // from this many active rows on, a projection CTA takes two weight tiles (-1: by shape)
     int tc_ksplit_cap = 1;          // bound the number of K ranges by the reduction traffic they add
     // sampling of the next token (greedy while sample_k <= 1)
     int sample_k = 0;
@@ -245,7 +245,13 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.n_pad = (mm + 15) / 16 * 16;
         p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
         p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
-        p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
+        // Two weight tiles per CTA share every activation tile.  Worth it exactly when the activation tiles are
+        // so wide that only one single-tile CTA would fit per SM anyway (from 96 rows): the tile pair halves the
+        // activation bytes an SM pulls from L2 per weight byte (config 3: -4 %; 115 rows: -16 % per step);
+        // below that, two single-tile CTAs per SM overlap each other's set-up and epilogue and win.
+        const int stage1 = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
+        if (c->tc_mt2_min_rows >= 0) p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
+        else p.mt = (3 * stage1 > c->tc_smem_kb * 1024) ? 2 : 1;
         if (epi == tc::kEpiSwiglu && n_out % 128) p.mt = 1;
         p.pair_rows = c->pair_rows;
         const int tile_rows = epi == tc::kEpiSwiglu ? (p.mt == 1 ? c->pair_rows : 128) : tc::kBlockM * p.mt;
@@ -898,7 +904,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
     else if (!std::strcmp(name, "fuse_rope")) c->fuse_rope = value != 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
-    else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : (1 << 30);
+    else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
     else return FIRST_E_ARG;
