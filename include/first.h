@@ -25,8 +25,9 @@
  *     ordinary host memory.  All tensors are owned by the caller and only borrowed:
  *     weights for the lifetime of the context, everything else for the call (the
  *     kernels of a call may still be running on `stream` when it returns).
- *   - The library allocates device memory only in first_create (its own scratch) and
- *     frees it in first_destroy.
+ *   - The library allocates device memory in first_create (its own scratch) and frees it in
+ *     first_destroy; the two later allocations are stated where they happen (first_prefill's
+ *     token scores, the internal logits row buffer of first_decode_step without `logits`).
  *   - Work is enqueued on the CUDA stream passed as `void *stream` (a cudaStream_t;
  *     NULL = the default stream).  Only first_set_mask and first_last_device_flags
  *     wait for the stream.
@@ -185,6 +186,42 @@ int first_prefill_route_static(int32_t layer, int32_t n_layers, int32_t d_model,
                                int32_t hidden_dtype, const int32_t *cu_seqlens, int32_t B, int64_t total_tokens,
                                const float *router_w, const float *router_b, float tau, int32_t mode,
                                uint8_t *mask, float *scores, uint32_t *flags, void *stream);
+
+/* Prompt phase of a ragged batch, in one call ("Inference for FiRST", item 1: no layer is skipped
+ * while the prompt is processed; "Adaptive Router Module": router l reads the hidden states that
+ * enter layer l, for every prompt token, and its mean over the sequence decides the layer for that
+ * sequence).  For every sequence b with prompt tokens[cu_seqlens[b] .. cu_seqlens[b+1]-1]:
+ * all layers run on all prompt tokens (causal attention inside the prompt), the rotated keys and
+ * the values of all n_b tokens are written to rows 0..n_b-1 of b's slab in EVERY layer,
+ * len[l][b] = n_b, pos[b] = n_b; router l's score rho[b][l] and mask[b][l] are formed as in
+ * first_prefill_route from the float32 residual stream entering layer l; logits[b] is the
+ * distribution after the last prompt token and next_tokens[b] its argmax (or a sampled token,
+ * see first_set_sampling) -- the first generated token, to be fed to the first first_decode_step.
+ * Whatever the slabs held before is overwritten from row 0.
+ *
+ * How it runs: the prompt tokens go through the kernels of first_decode_step in chunks of
+ * min(max_batch, 256) tokens, each token a row of its own (its slab is its sequence's slab, its
+ * cache length its position), so a context meant for prefill should be created with max_batch
+ * of 256 or more.  Weights are streamed once per chunk.  The chunks run without CUDA graphs.
+ *   tokens        dev int32 [total], total = cu_seqlens[B]
+ *   cu_seqlens    HOST int32 [B+1], cu_seqlens[0] = 0, strictly increasing (no empty prompt);
+ *                 every prompt at most max_tokens_per_seq tokens, B at most max_batch
+ *   kv            host struct, per_layer = 0 (FIRST_E_UNSUPPORTED otherwise); a slab shorter than
+ *                 its prompt sets FIRST_FLAG_KV_FULL and keeps only the tokens that fit
+ *   router_w      dev float32 [n_layers][d_model], or NULL: no routing, mask/scores untouched
+ *   router_b      dev float32 [n_layers] or NULL (the paper's routers have no bias)
+ *   tau, mode     as in first_prefill_route
+ *   mask          dev uint8 [B][n_layers] (required with router_w); scores dev float32 [B][n_layers] or NULL
+ *   logits        dev float32 [B][vocab] or NULL;  next_tokens  dev int32 [B] or NULL
+ * The call waits for the stream before it returns.  It replaces the context's plan: call
+ * first_set_mask (with the mask it produced, or any other) before the next first_decode_step.
+ * With routers, the first call allocates n_layers*total float32 of token scores (kept, and
+ * grown when a later call needs more); must not be called while `stream` is being captured.
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_UNSUPPORTED, FIRST_E_STATE (stream capture),
+ * FIRST_E_CUDA; device flags for a full slab or a bad token id. */
+int first_prefill(first_ctx *ctx, const int32_t *tokens, const int32_t *cu_seqlens, int32_t B,
+                  const first_kv_cache *kv, const float *router_w, const float *router_b, float tau, int32_t mode,
+                  uint8_t *mask, float *scores, float *logits, int32_t *next_tokens, void *stream);
 
 /* Fix the skip mask of the current batch and build, per layer, the ascending list of
  * rows that keep it (one decision per sequence per layer, "Adaptive Router Module";

@@ -65,6 +65,10 @@ def lib():
                                                  C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_float, C.c_int32,
                                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_prefill_route_static.restype = C.c_int
+        L.first_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(KVCacheC), C.c_void_p,
+                                    C.c_void_p, C.c_float, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_void_p]
+        L.first_prefill.restype = C.c_int
         L.first_set_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.first_get_plan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(KVCacheC), C.c_void_p, C.c_void_p,
@@ -198,6 +202,20 @@ def first_prefill_route_static(layer, n_layers, hidden, cu_seqlens, router_w, ro
         raise FirstError(rc, "first_prefill_route_static")
 
 
+def first_prefill(h, tokens, cu_seqlens, kv: KVCache, router_w=None, router_b=None, tau=0.5, mode=0, mask=None,
+                  scores=None, logits=None, next_tokens=None, stream=None):
+    """Whole prompt phase of a ragged batch; cu_seqlens is a HOST int32 array (numpy or a CPU tensor)."""
+    import numpy as np
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens), dtype=np.int32)
+    rc = lib().first_prefill(h, _dev(tokens, torch.int32, "tokens"), cu.ctypes.data, cu.size - 1, C.byref(kv.c),
+                             _dev(router_w, torch.float32, "router_w"), _dev(router_b, torch.float32, "router_b"),
+                             float(tau), int(mode), _dev(mask, torch.uint8, "mask"),
+                             _dev(scores, torch.float32, "scores"), _dev(logits, torch.float32, "logits"),
+                             _dev(next_tokens, torch.int32, "next_tokens"), _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_prefill")
+
+
 def first_set_mask(h, mask, stream=None):
     rc = lib().first_set_mask(h, _dev(mask, torch.uint8, "mask"), mask.shape[0], _stream(stream))
     if rc:
@@ -297,6 +315,11 @@ class FirstContext:
 
     def prefill_route(self, layer, hidden, cu_seqlens, router_w, router_b, tau, mode, mask, scores=None, stream=None):
         first_prefill_route(self.h, layer, hidden, cu_seqlens, router_w, router_b, tau, mode, mask, scores, stream)
+
+    def prefill(self, tokens, cu_seqlens, kv, router_w=None, router_b=None, tau=0.5, mode=0, mask=None, scores=None,
+                logits=None, next_tokens=None, stream=None):
+        first_prefill(self.h, tokens, cu_seqlens, kv, router_w, router_b, tau, mode, mask, scores, logits,
+                      next_tokens, stream)
 
     def set_mask(self, mask, stream=None):
         first_set_mask(self.h, mask, stream)

@@ -14,6 +14,7 @@
 #include "first.h"
 #include "gemm_tc.cuh"
 #include "gemv.cuh"
+#include "prefill.cuh"
 #include "router.cuh"
 #include "step.cuh"
 
@@ -31,11 +32,11 @@ using namespace first;
 static thread_local char g_last_cuda_error[256] = "";
 
 enum KernelClass { kClsStepBegin = 0, kClsRmsnorm, kClsGemv, kClsGemmTc, kClsRopeAppend, kClsAttn, kClsAttnCombine,
-                   kClsSiluMul, kClsStepEnd, kClsRouterScores, kClsRouterFinalize, kClsPlan, kNumClasses };
+                   kClsSiluMul, kClsStepEnd, kClsRouterScores, kClsRouterFinalize, kClsPlan, kClsPrefillAux, kNumClasses };
 static const char* const kClassNames[kNumClasses] = {"step_begin", "rmsnorm_rows", "gemv_rows", "gemm_tc",
                                                      "rope_append", "attn_split", "attn_combine", "silu_mul",
                                                      "step_end", "router_token_scores", "router_finalize",
-                                                     "plan_compact"};
+                                                     "plan_compact", "prefill_aux"};
 
 struct first_ctx {
     first_model_desc d{};
@@ -103,6 +104,22 @@ struct first_ctx {
     int sample_k = 0;
     float sample_inv_T = 1.f;
     const float* sample_u = nullptr;
+    // batched prefill: per-row tables of a chunk (each prompt token is a row), an all-keep mask, the residual of
+    // every sequence's last prompt token, and (allocated on first use) the per-layer token scores of the routers
+    int32_t *pf_cu = nullptr, *pf_tok = nullptr, *pf_cap = nullptr, *pf_pos = nullptr, *pf_len = nullptr;
+    int64_t* pf_off = nullptr;
+    uint8_t* pf_ones = nullptr;
+    float *x_last = nullptr, *pf_score = nullptr;
+    int64_t pf_score_cap = 0;
+};
+
+// What a chunk of a batched prefill does beyond a decode step: router l scores the chunk's rows as they
+// enter layer l (token scores of layer l at tokscore + l*stride + g0), and the step ends after the last layer.
+struct PrefillHook {
+    const float *router_w, *router_b;  // dev [L][D], dev [L] or nullptr
+    int mode;
+    float* tokscore;
+    int64_t stride, g0;
 };
 
 constexpr int kSimpleSplitsMax = 16;
@@ -478,10 +495,13 @@ int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUt
     return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
 }
 
+template <typename WT>
+int logits_tail(first_ctx* c, cudaStream_t st, int B, float* logits, int32_t* next_tokens, int32_t* pos);
+
 // The whole step, for one weight/cache element type.
 template <typename WT>
 int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* kv, float* logits,
-                     int32_t* next_tokens, float* layer_inputs, cudaStream_t st) {
+                     int32_t* next_tokens, float* layer_inputs, cudaStream_t st, const PrefillHook* ph = nullptr) {
     const first_model_desc& d = c->d;
     const int B = c->B, D = d.d_model, F = d.ffn_dim, V = d.vocab, L = d.n_layers, hd = d.head_dim;
     constexpr bool kBf16 = std::is_same<WT, __nv_bfloat16>::value;
@@ -504,6 +524,15 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         if (layer_inputs) {
             CU_TRY(cudaMemcpyAsync(layer_inputs + (size_t)l * B * D, c->x, (size_t)B * D * sizeof(float),
                                    cudaMemcpyDeviceToDevice, st));
+            c->pdl_next = false;
+        }
+        if (ph && ph->router_w) {  // prefill: router l reads the rows entering layer l
+            const int blocks = std::min((B + 7) / 8, c->n_sm * 8);
+            FIRST_LAUNCH(kClsRouterScores, (router_token_scores<float><<<blocks, 256, (size_t)D * sizeof(float), st>>>(
+                                               c->x, (int64_t)B, D, ph->router_w + (size_t)l * D,
+                                               ph->router_b ? ph->router_b + l : nullptr, ph->mode,
+                                               ph->tokscore + (size_t)l * ph->stride + ph->g0)));
+            if ((rc = check_launch(c))) return rc;
             c->pdl_next = false;
         }
         const int m = c->cnt_h[l];
@@ -571,6 +600,20 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                               c->x, D, idx)))
             return rc;
     }
+    if (ph) return FIRST_OK;  // a prefill chunk ends here: logits are taken once, from the last prompt tokens
+    return logits_tail<WT>(c, st, B, logits, next_tokens, kv->pos);
+}
+
+// Final norm, lm_head and next token of rows 0..B-1 of the residual stream; pos += 1.
+template <typename WT>
+int logits_tail(first_ctx* c, cudaStream_t st, int B, float* logits, int32_t* next_tokens, int32_t* pos) {
+    const first_model_desc& d = c->d;
+    const int D = d.d_model, V = d.vocab;
+    constexpr bool kBf16 = std::is_same<WT, __nv_bfloat16>::value;
+    const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 0;
+    auto tc_for = [&](int m) { return kBf16 && c->tc_ready && m > gemv_max; };
+    const int norm_threads = std::max(32, std::min(1024, (D / 4 + 31) / 32 * 32));
+    int rc;
     float* lg = logits ? logits : (next_tokens ? c->logits_int : nullptr);
     if (lg) {
         const bool t = tc_for(B);
@@ -584,8 +627,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     }
     if (next_tokens && lg && c->sample_k > 1)
         return launch_k(c, st, kClsStepEnd, step_end_sample, dim3(B), dim3(1024), 0, lg, V, c->sample_k, c->sample_inv_T,
-                        c->sample_u, next_tokens, kv->pos);
-    return launch_k(c, st, kClsStepEnd, step_end, dim3(B), dim3(1024), 0, lg, V, next_tokens, kv->pos);
+                        c->sample_u, next_tokens, pos);
+    return launch_k(c, st, kClsStepEnd, step_end, dim3(B), dim3(1024), 0, lg, V, next_tokens, pos);
 }
 
 }  // namespace
@@ -664,6 +707,12 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)) || (rc = dev_alloc(&c->rowinfo, MB)))
         return fail(rc);
     if (cudaMemset(c->ticket, 0, MB * d.n_kv_heads * sizeof(uint32_t)) != cudaSuccess) return fail(FIRST_E_CUDA);
+    if ((rc = dev_alloc(&c->pf_cu, MB + 1)) || (rc = dev_alloc(&c->pf_tok, MB)) || (rc = dev_alloc(&c->pf_cap, MB)) ||
+        (rc = dev_alloc(&c->pf_pos, MB)) || (rc = dev_alloc(&c->pf_len, MB * d.n_layers)) ||
+        (rc = dev_alloc(&c->pf_off, MB)) || (rc = dev_alloc(&c->pf_ones, MB * d.n_layers)) ||
+        (rc = dev_alloc(&c->x_last, MB * d.d_model)))
+        return fail(rc);
+    if (cudaMemset(c->pf_ones, 1, MB * d.n_layers) != cudaSuccess) return fail(FIRST_E_CUDA);
     if (d.dtype == FIRST_DTYPE_BF16) {
         if ((rc = dev_alloc(&c->xh, MB * xw)) || (rc = dev_alloc(&c->xl, MB * xw)) ||
             (rc = dev_alloc(&c->acth, MB * d.ffn_dim)) || (rc = dev_alloc(&c->actl, MB * d.ffn_dim)))
@@ -685,7 +734,8 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
 int first_destroy(first_ctx* c) {
     if (!c) return FIRST_OK;
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
-                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket, c->rowinfo};
+                    c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket, c->rowinfo,
+                    c->pf_cu, c->pf_tok, c->pf_cap, c->pf_pos, c->pf_len, c->pf_off, c->pf_ones, c->x_last, c->pf_score};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -826,6 +876,102 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     g->last_use = ++c->use_clock;
     CU_TRY(cudaGraphLaunch(g->exec, st));
     c->launches += g->n_launches;
+    return FIRST_OK;
+}
+
+int first_prefill(first_ctx* c, const int32_t* tokens, const int32_t* cu_seqlens, int32_t B, const first_kv_cache* kv,
+                  const float* router_w, const float* router_b, float tau, int32_t mode, uint8_t* mask, float* scores,
+                  float* logits, int32_t* next_tokens, void* stream) {
+    if (!c || !tokens || !cu_seqlens || !kv || B <= 0) return FIRST_E_ARG;
+    if (!kv->k || !kv->v || !kv->slab_off || !kv->slab_cap || !kv->len || !kv->pos) return FIRST_E_ARG;
+    if (kv->per_layer) return FIRST_E_UNSUPPORTED;  // the prompt fills every layer: one table serves them all
+    if (kv->cap_total <= 0) return FIRST_E_ARG;
+    const first_model_desc& d = c->d;
+    const int L = d.n_layers, D = d.d_model;
+    for (int l = 0; l < L; ++l)
+        if (!kv->k[l] || !kv->v[l]) return FIRST_E_ARG;
+    if (router_w) {
+        if (!mask) return FIRST_E_ARG;
+        if (mode != FIRST_ROUTER_MEAN_OF_SIGMOID && mode != FIRST_ROUTER_SIGMOID_OF_MEAN) return FIRST_E_ARG;
+        if (!(tau > 0.f && tau < 1.f)) return FIRST_E_ARG;
+        if (D > 12288) return FIRST_E_UNSUPPORTED;
+    }
+    if (B > d.max_batch) return FIRST_E_CAPACITY;
+    if (cu_seqlens[0] != 0) return FIRST_E_ARG;
+    for (int b = 0; b < B; ++b) {
+        const int64_t n = (int64_t)cu_seqlens[b + 1] - cu_seqlens[b];
+        if (n <= 0) return FIRST_E_ARG;  // every sequence brings at least one prompt token
+        if (n > d.max_tokens_per_seq) return FIRST_E_CAPACITY;
+    }
+    const int64_t total = cu_seqlens[B];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_TRY(cudaStreamIsCapturing(st, &cap));
+    if (cap != cudaStreamCaptureStatusNone) return FIRST_E_STATE;  // this call waits for the stream
+    if (router_w && (int64_t)L * total > c->pf_score_cap) {
+        if (c->pf_score) cudaFree(c->pf_score);
+        c->pf_score = nullptr;
+        c->pf_score_cap = 0;
+        int rc = dev_alloc(&c->pf_score, (size_t)L * total);
+        if (rc) return rc;
+        c->pf_score_cap = (int64_t)L * total;
+    }
+    if (!logits && next_tokens && !c->logits_int) {
+        int rc = dev_alloc(&c->logits_int, (size_t)d.max_batch * d.vocab);
+        if (rc) return rc;
+    }
+    CU_TRY(cudaMemcpyAsync(c->pf_cu, cu_seqlens, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, st));
+
+    // Each prompt token is a row of its own for the step kernels, so the rotate-and-append kernel must finish
+    // a chunk's keys and values before attention starts (a row attends over earlier rows of its own chunk).
+    struct Restore {
+        first_ctx* c; int fuse_rope;
+        ~Restore() { c->fuse_rope = fuse_rope; c->has_mask = false; }
+    } restore{c, c->fuse_rope};
+    c->fuse_rope = 0;
+
+    first_kv_cache vkv = *kv;
+    vkv.slab_off = c->pf_off;
+    vkv.slab_cap = c->pf_cap;
+    vkv.len = c->pf_len;
+    vkv.pos = c->pf_pos;
+    const int R = (int)std::min<int64_t>(std::min(d.max_batch, 256), total);
+    int plan_rows = 0, rc;
+    for (int64_t g0 = 0; g0 < total; g0 += R) {
+        const int rows = (int)std::min<int64_t>(R, total - g0);
+        if (rows != plan_rows) {  // all-keep plan over this many rows (at most twice per call)
+            if ((rc = first_set_mask(c, c->pf_ones, rows, stream))) return rc;
+            plan_rows = rows;
+        }
+        FIRST_LAUNCH(kClsPrefillAux, (prefill_rows<<<(rows + 127) / 128, 128, 0, st>>>(
+                                         tokens, c->pf_cu, B, (int)g0, rows, L, kv->slab_off, kv->slab_cap, c->pf_tok,
+                                         c->pf_off, c->pf_cap, c->pf_pos, c->pf_len)));
+        if ((rc = check_launch(c))) return rc;
+        const PrefillHook ph{router_w, router_b, mode, c->pf_score, total, g0};
+        rc = d.dtype == FIRST_DTYPE_BF16
+                 ? decode_step_impl<__nv_bfloat16>(c, c->pf_tok, &vkv, nullptr, nullptr, nullptr, st, &ph)
+                 : decode_step_impl<float>(c, c->pf_tok, &vkv, nullptr, nullptr, nullptr, st, &ph);
+        if (rc) return rc;
+        FIRST_LAUNCH(kClsPrefillAux, (prefill_keep_last<<<rows, 256, 0, st>>>(c->x, c->pf_cu, B, (int)g0, D, c->x_last)));
+        if ((rc = check_launch(c))) return rc;
+    }
+    if (router_w)
+        for (int l = 0; l < L; ++l) {
+            FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->pf_score + (size_t)l * total, c->pf_cu, L, l,
+                                                                                 mode, tau, mask, scores, c->flags)));
+            if ((rc = check_launch(c))) return rc;
+        }
+    FIRST_LAUNCH(kClsPrefillAux, (prefill_finish<<<(B + 127) / 128, 128, 0, st>>>(c->pf_cu, B, L, kv->slab_cap, kv->len, kv->pos)));
+    if ((rc = check_launch(c))) return rc;
+    if (logits || next_tokens) {
+        CU_TRY(cudaMemcpyAsync(c->x, c->x_last, (size_t)B * D * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        c->pdl_next = false;
+        // the tail advances a position counter: hand it the chunk table, pos[] already holds the prompt lengths
+        rc = d.dtype == FIRST_DTYPE_BF16 ? logits_tail<__nv_bfloat16>(c, st, B, logits, next_tokens, c->pf_pos)
+                                         : logits_tail<float>(c, st, B, logits, next_tokens, c->pf_pos);
+        if (rc) return rc;
+    }
+    CU_TRY(cudaStreamSynchronize(st));  // cu_seqlens was read from host memory; the plan of the last chunk is dropped
     return FIRST_OK;
 }
 

@@ -33,6 +33,7 @@ def test_status_strings_and_null_argument_errors_need_no_gpu():
     assert L.first_decode_step(None, None, None, None, None, None, None) == -1
     assert L.first_set_mask(None, None, 1, None) == -1
     assert L.first_prefill_route(None, 0, None, 0, None, 1, 1, None, None, 0.5, 0, None, None, None) == -1
+    assert L.first_prefill(None, None, None, 1, None, None, None, 0.5, 0, None, None, None, None, None) == -1
     assert L.first_destroy(None) == 0
 
 

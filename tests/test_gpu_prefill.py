@@ -1,0 +1,170 @@
+"""first_prefill (whole prompt phase in one call) vs the host oracle's prefill, through the C ABI (B200 only).
+
+"Inference for FiRST": (1) the prompt runs through every layer, (2) the routers' decisions on the
+prompt are then fixed for the decode steps.  Checked here: keys/values of every layer, len/pos,
+first-token logits, router scores and masks (bit-exact), and routed decode steps that continue
+from the prefilled caches.
+"""
+import numpy as np
+import pytest
+
+import first_inputs as fi
+import oracle
+from harness import GpuKV, calibrate_router, gpu_weights, logits_check, oracle_model, to_dev
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = 0, 1
+SMALL_GQA = fi.ModelShape(3, 256, 8, 2, 64, 512, 2048, 500000.0)
+
+
+def _ctx(shape, bf16, max_batch, max_tokens, w):
+    from paper_2410_12513_b200 import FirstContext
+    return FirstContext(shape, BF16 if bf16 else F32, max_batch, max_tokens, gpu_weights(w))
+
+
+def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_tol, options=None):
+    """Oracle prefill per sequence -> routers calibrated on its layer inputs -> one first_prefill
+    call on the GPU -> everything it leaves behind compared -> `steps` routed decode steps."""
+    import torch
+    B, L = len(lens), shape.n_layers
+    w = fi.make_weights(shape, seed, bf16)
+    om = oracle_model(shape, w)
+    prompts = [fi.tokens(shape, int(n), seed, f"prompt{b}") for b, n in enumerate(lens)]
+    caps = [int(n) + steps + (3 if b == 0 else 0) for b, n in enumerate(lens)]
+    okv = oracle.OracleKV(om.shape, caps)
+    pre = [oracle.prefill(om, okv, b, prompts[b]) for b in range(B)]
+    target = fi.mask_bernoulli(B, L, keep_p, seed + 7)
+    routers, rho = [], []
+    for l in range(L):
+        rw, r = calibrate_router([pre[b]["router_in"][l] for b in range(B)], target[:, l], mode, l)
+        routers.append(rw)
+        rho.append(r)
+    rho = np.stack(rho, 1)  # [B][L]
+
+    gkv = GpuKV(shape, caps, bf16)
+    ctx = _ctx(shape, bf16, max_batch, max(caps), w)
+    for k, v in (options or {}).items():
+        ctx.set_option(k, v)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    toks = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
+    mask = torch.full((B, L), 7, dtype=torch.uint8, device="cuda")
+    scores = torch.zeros((B, L), dtype=torch.float32, device="cuda")
+    logits = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda")
+    nxt = torch.empty((B,), dtype=torch.int32, device="cuda")
+    ctx.prefill(toks, cu, gkv.c, to_dev(np.stack(routers), False), None, 0.5, mode, mask, scores, logits, nxt)
+    assert ctx.device_flags() == 0
+
+    # bookkeeping and caches: every layer holds the whole prompt
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
+    assert np.array_equal(gkv.pos.cpu().numpy(), okv.pos)
+    tol = 2e-2 if bf16 else 1e-4
+    for l in range(L):
+        for b in range(B):
+            n = int(lens[b])
+            k1, v1 = gkv.rows_host(l, b)
+            ko, vo = okv.rows(l, b)
+            assert np.abs(k1[:n] - ko[:n]).max() <= tol * max(1.0, np.abs(ko[:n]).max()), (l, b)
+            assert np.abs(v1[:n] - vo[:n]).max() <= tol * max(1.0, np.abs(vo[:n]).max()), (l, b)
+            assert not k1[n:].any() and not v1[n:].any()  # nothing written past the prompt
+    # first-token logits and greedy token
+    ref0 = np.stack([pre[b]["logits"][0] if pre[b]["logits"].ndim > 1 else pre[b]["logits"] for b in range(B)])
+    got0 = logits.cpu().numpy()
+    err, agree = logits_check(got0, ref0)
+    assert err.max() <= rel_tol, err.max()
+    assert np.array_equal(nxt.cpu().numpy(), got0.argmax(-1).astype(np.int32))
+    # routers: masks bit-exact, scores close
+    assert np.array_equal(mask.cpu().numpy(), target)
+    assert np.abs(scores.cpu().numpy() - rho).max() <= (5e-3 if bf16 else 1e-5)
+
+    # the decode steps that follow obey the masks and continue from these caches
+    with pytest.raises(Exception):
+        ctx.decode_step(nxt, gkv.c, logits)  # the prefill dropped the plan: a mask must be set first
+    ctx.set_mask(mask)
+    toks_t = oracle.argmax(ref0)
+    for t in range(steps):
+        ref = oracle.decode_step(om, toks_t, target, okv)
+        ctx.decode_step(torch.from_numpy(toks_t).cuda(), gkv.c, logits)
+        err, agree = logits_check(logits.cpu().numpy(), ref)
+        assert err.max() <= rel_tol, (t, err.max())
+        toks_t = oracle.argmax(ref)
+    assert ctx.device_flags() == 0
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
+    assert np.array_equal(gkv.pos.cpu().numpy(), okv.pos)
+    return err
+
+
+def test_prefill_config0_chunks_cross_sequence_boundaries():
+    """Tiny fp32 decoder, batch 2, prompts of 32 tokens (config 0), pooled-sigmoid routers; chunks of
+    24 rows: 24 + 24 + 16, the second one holding the end of sequence 0 and the start of sequence 1."""
+    _prefill_case(fi.TINY, False, [32, 32], 24, 4, 0, 1, 0.6, 1e-4)
+
+
+@pytest.mark.parametrize("max_batch", [5, 64, 300])
+def test_prefill_f32_ragged(max_batch):
+    """Ragged prompts (one of a single token), the paper's router order, three chunk sizes: a chunk per
+    few tokens, chunks of 64, and one chunk shorter than the 256-row limit for the whole batch."""
+    _prefill_case(fi.TINY, False, [1, 17, 64, 9, 40], max_batch, 3, 3, 0, 0.5, 1e-4)
+
+
+@pytest.mark.parametrize("max_batch", [48, 256])
+def test_prefill_bf16_gqa_ragged(max_batch):
+    """bfloat16 weights and caches, 4 query heads per KV head, head_dim 64: tensor-core projections and
+    the tuned attention kernel on chunk rows."""
+    _prefill_case(SMALL_GQA, True, [8, 200, 77, 130, 1], max_batch, 3, 5, 0, 0.6, 2e-2)
+
+
+def test_prefill_bf16_general_kernels_by_option():
+    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"attn_simple": 1, "max_gemv_rows": 1024})
+
+
+def test_prefill_without_routers_and_outputs():
+    """router_w = NULL leaves mask and scores alone; logits/next_tokens may be omitted."""
+    import torch
+    shape, lens = fi.TINY, [12, 5]
+    w = fi.make_weights(shape, 1, False)
+    om = oracle_model(shape, w)
+    prompts = [fi.tokens(shape, n, 1, f"p{b}") for b, n in enumerate(lens)]
+    okv = oracle.OracleKV(om.shape, [20, 20])
+    for b in range(2):
+        oracle.prefill(om, okv, b, prompts[b], want_router_in=False)
+    gkv = GpuKV(shape, [20, 20], False)
+    ctx = _ctx(shape, False, 8, 20, w)
+    cu = np.array([0, 12, 17], np.int32)
+    ctx.prefill(torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda(), cu, gkv.c)
+    assert ctx.device_flags() == 0
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len) and np.array_equal(gkv.pos.cpu().numpy(), okv.pos)
+    for l in range(shape.n_layers):
+        for b in range(2):
+            k1, v1 = gkv.rows_host(l, b)
+            ko, vo = okv.rows(l, b)
+            assert np.abs(k1 - ko).max() <= 1e-4 and np.abs(v1 - vo).max() <= 1e-4
+
+
+def test_prefill_argument_errors_and_short_slab():
+    import torch
+    from paper_2410_12513_b200 import FirstError
+    shape = fi.TINY
+    w = fi.make_weights(shape, 2, False)
+    ctx = _ctx(shape, False, 4, 16, w)
+    gkv = GpuKV(shape, [16, 6], False)
+    toks = torch.zeros((64,), dtype=torch.int32, device="cuda")
+
+    def status(cu, kv=gkv.c):
+        with pytest.raises(FirstError) as e:
+            ctx.prefill(toks, np.asarray(cu, np.int32), kv)
+        return e.value.status
+
+    assert status([0, 4, 4]) == -1            # empty prompt
+    assert status([1, 4, 6]) == -1            # cu_seqlens[0] != 0
+    assert status([0, 17, 20]) == -4          # prompt longer than max_tokens_per_seq
+    assert status([0, 1, 2, 3, 4, 5]) == -4   # batch larger than max_batch
+    # a slab shorter than its prompt: flagged, the tokens that fit are kept, the neighbouring slab is not touched
+    guard = GpuKV(shape, [6, 16], False)
+    ctx.prefill(toks, np.array([0, 8, 11], np.int32), guard.c)
+    assert ctx.device_flags() == 1
+    assert guard.len.cpu().numpy().tolist() == [[6, 3]] * shape.n_layers
+    assert guard.pos.cpu().numpy().tolist() == [8, 3]
+    for l in range(shape.n_layers):
+        k1, v1 = guard.rows_host(l, 1)
+        assert k1[:3].any() and not k1[3:].any() and not v1[3:].any()
