@@ -217,6 +217,45 @@ def run_reference(args, wl, shape, mask, lens):
     print(json.dumps(out))
 
 
+def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, max_tokens=40000):
+    """The prompt phase that precedes the timed decode steps, on this workload's prompts (the first sequences of
+    the batch up to `max_tokens` prompt tokens): one first_prefill call with routers, timed with CUDA events.
+    Reported beside the decode metric, not part of it; it overwrites the stand-in caches, so it runs last."""
+    s, L = shape, shape.n_layers
+    nb = int(max(1, np.searchsorted(np.cumsum(lens), max_tokens, side="right")))
+    pl = lens[:nb]
+    total = int(pl.sum())
+    ctx = FirstContext(shape, 1, max(256, nb), int(caps.max()), weights)
+    cu = np.concatenate([[0], np.cumsum(pl)]).astype(np.int32)
+    toks = torch.from_numpy(fi.tokens(shape, total, 11)).to(dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(99)
+    rw = 0.02 * torch.randn((L, s.d_model), device=dev, generator=g)
+    mask = torch.zeros((nb, L), dtype=torch.uint8, device=dev)
+    nxt = torch.empty((nb,), dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    ctx.prefill(toks[:int(cu[1])], cu[:2], kv, rw, None, 0.5, 0, mask[:1], None, None, nxt[:1])  # warm-up: one prompt
+    torch.cuda.synchronize()
+    l0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    ctx.prefill(toks, cu, kv, rw, None, 0.5, 0, mask, None, None, nxt)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    flags = ctx.device_flags()
+    if flags:
+        raise RuntimeError(f"device flags set during the prefill leg: {flags}")
+    proj = 2.0 * s.layer_params() * L * total + 2.0 * s.vocab * s.d_model * nb
+    attn = float(sum(2.0 * int(n) * int(n) * s.head_dim * s.n_q_heads * L for n in pl))
+    tf = (proj + attn) / ms / 1e9
+    pk = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    return {"sequences": nb, "prompt_tokens": total, "ms": ms, "tokens_per_s": total / ms * 1e3,
+            "model_tflops": tf, "frac_of_bf16_sustained_peak": tf / pk, "gpu_launches": int(ctx.launch_count() - l0),
+            "chunk_rows": 256, "kept_fraction_routed": float(mask.float().mean().item()),
+            "note": "prompt tokens as rows of the decode-step kernels, 256 per chunk; weights streamed once per chunk"}
+
+
 # ----------------------------------------------------------------------------- CUDA arm
 def run_cuda(args, wl, shape, mask, lens):
     import torch
@@ -464,6 +503,8 @@ def run_cuda(args, wl, shape, mask, lens):
                      "bytes_ratio_routed_over_dense": bm["full"] / bm_dense["full"]},
            "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
            "kernel_ms_per_step": cls_ms, "route": route}
+    if not args.no_prefill:
+        out["prefill"] = prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks)
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5, rows=min(B, 32), layers=4)
         out["cpu_baseline"].pop("ms_per_step", None)
@@ -482,6 +523,7 @@ def main():
     ap.add_argument("--mask", default=None, help="override: dense | aligned:F | independent:F | fraction:LO:HI | bernoulli:P | unified:EVERY | random:F")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-route", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the prompt-phase leg (first_prefill on this workload's prompts)")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (A/B runs)")
     ap.add_argument("--layers", type=int, default=None,
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")

@@ -112,23 +112,47 @@ def test_config3_shape_b256_heterogeneous_masks(w8b):
     _stand_in_case(shape, w, gw, om, lens, mask, list(range(0, B, 32)), 2, 23, "config3")
 
 
+_cfg1 = {}
+
+
+def _clone_okv(om, src):
+    dst = oracle.OracleKV(om.shape, src.slab_cap)
+    for l in range(src.L):
+        dst.k[l][:] = src.k[l]
+        dst.v[l][:] = src.v[l]
+    dst.len[:], dst.pos[:] = src.len, src.pos
+    return dst
+
+
+def _config1_oracle():
+    """Oracle side of config 1, built once for the tests below: weights, the oracle's prefill of the
+    512-token prompt (caches, layer inputs, first logits), routers calibrated on its layer inputs."""
+    if not _cfg1:
+        shape, n, S = fi.LLAMA_1B, 512, 256
+        w = fi.make_weights(shape, 1000, True)
+        om = oracle_model(shape, w)
+        prompt = fi.tokens(shape, n, 1000, "prompt")
+        okv = oracle.OracleKV(om.shape, [n + S])
+        pre = oracle.prefill(om, okv, 0, prompt)
+        target = fi.mask_aligned(1, shape.n_layers, 0.25)  # ~25 % of the layers skipped
+        routers = [calibrate_router([pre["router_in"][l]], target[:, l], 1, l)[0] for l in range(shape.n_layers)]
+        _cfg1.update(shape=shape, n=n, S=S, w=w, om=om, prompt=prompt, okv=okv, pre=pre, target=target,
+                     routers=routers, gw=gpu_weights(w))
+    return _cfg1
+
+
 def test_config1_shape_prefill_route_decode():
     """Llama-3.2-1B shape, batch 1, prompt 512: GPU prefill token by token (all-keep), routers on
     the captured layer inputs (masks bit-exact vs the oracle on its own prefill), then routed
     greedy decode, teacher-forced, every step checked."""
     import torch
     from paper_2410_12513_b200 import FirstContext
-    shape, n, S = fi.LLAMA_1B, 512, 256
+    c = _config1_oracle()
+    shape, n, S, om, prompt, pre, target, routers = (c[k] for k in ("shape", "n", "S", "om", "prompt", "pre", "target", "routers"))
+    okv = _clone_okv(om, c["okv"])
     L, D = shape.n_layers, shape.d_model
-    w = fi.make_weights(shape, 1000, True)
-    om = oracle_model(shape, w)
-    prompt = fi.tokens(shape, n, 1000, "prompt")
-    okv = oracle.OracleKV(om.shape, [n + S])
-    pre = oracle.prefill(om, okv, 0, prompt)
-    target = fi.mask_aligned(1, L, 0.25)  # ~25 % of the layers skipped
-    routers = [calibrate_router([pre["router_in"][l]], target[:, l], 1, l)[0] for l in range(L)]
     gkv = GpuKV(shape, [n + S], True)
-    ctx = FirstContext(shape, 1, 1, n + S, gpu_weights(w))
+    ctx = FirstContext(shape, 1, 1, n + S, c["gw"])
     ctx.set_mask(torch.ones((1, L), dtype=torch.uint8, device="cuda"))
     li = torch.empty((n, L, 1, D), dtype=torch.float32, device="cuda")
     logits = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
@@ -155,6 +179,48 @@ def test_config1_shape_prefill_route_decode():
         got = logits.cpu().numpy()
         err, agree = logits_check(got, ref)
         _account(err, agree, got, ref, "config1")
+        toks = oracle.argmax(ref)
+    assert ctx.device_flags() == 0
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
+
+
+def test_config1_shape_one_call_prefill():
+    """Config 1 again with the prompt phase as ONE first_prefill call (two chunks of 256 prompt tokens):
+    caches of all 16 layers, first logits and router masks against the oracle's prefill, then routed
+    decode steps from those caches, teacher-forced."""
+    import torch
+    from paper_2410_12513_b200 import FirstContext
+    c = _config1_oracle()
+    shape, n, S, om, prompt, pre, target, routers = (c[k] for k in ("shape", "n", "S", "om", "prompt", "pre", "target", "routers"))
+    okv = _clone_okv(om, c["okv"])
+    L = shape.n_layers
+    gkv = GpuKV(shape, [n + S], True)
+    ctx = FirstContext(shape, 1, 256, n + S, c["gw"])
+    mask = torch.zeros((1, L), dtype=torch.uint8, device="cuda")
+    logits = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+    nxt = torch.empty((1,), dtype=torch.int32, device="cuda")
+    ctx.prefill(torch.from_numpy(prompt.astype(np.int32)).cuda(), np.array([0, n], np.int32), gkv.c,
+                to_dev(np.stack(routers), False), None, 0.5, 1, mask, None, logits, nxt)
+    assert ctx.device_flags() == 0
+    got = logits.cpu().numpy()
+    err, agree = logits_check(got, pre["logits"])
+    _account(err, agree, got, pre["logits"], "config1_prefill")
+    assert int(nxt.item()) == int(got.argmax(-1)[0])
+    assert np.array_equal(mask.cpu().numpy(), target)
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len) and np.array_equal(gkv.pos.cpu().numpy(), okv.pos)
+    for l in range(L):
+        k1, v1 = gkv.rows_host(l, 0)
+        ko, vo = okv.rows(l, 0)
+        assert np.abs(k1[:n] - ko[:n]).max() <= 2e-2 * max(1.0, np.abs(ko[:n]).max()), l
+        assert np.abs(v1[:n] - vo[:n]).max() <= 2e-2 * max(1.0, np.abs(vo[:n]).max()), l
+    ctx.set_mask(mask)
+    toks = oracle.argmax(pre["logits"])
+    for t in range(32):
+        ref = oracle.decode_step(om, toks, target, okv)
+        ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits)
+        got = logits.cpu().numpy()
+        err, agree = logits_check(got, ref)
+        _account(err, agree, got, ref, "config1_prefill")
         toks = oracle.argmax(ref)
     assert ctx.device_flags() == 0
     assert np.array_equal(gkv.len.cpu().numpy(), okv.len)
