@@ -217,7 +217,7 @@ def run_reference(args, wl, shape, mask, lens):
     print(json.dumps(out))
 
 
-def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, max_tokens=40000):
+def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, max_tokens=40000, opts=()):
     """The prompt phase that precedes the timed decode steps, on this workload's prompts (the first sequences of
     the batch up to `max_tokens` prompt tokens): one first_prefill call with routers, timed with CUDA events.
     Reported beside the decode metric, not part of it; it overwrites the stand-in caches, so it runs last."""
@@ -226,6 +226,9 @@ def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks,
     pl = lens[:nb]
     total = int(pl.sum())
     ctx = FirstContext(shape, 1, max(256, nb), int(caps.max()), weights)
+    for o in opts:
+        name, val = o.split("=")
+        ctx.set_option(name, int(val))
     cu = np.concatenate([[0], np.cumsum(pl)]).astype(np.int32)
     toks = torch.from_numpy(fi.tokens(shape, total, 11)).to(dev)
     g = torch.Generator(device=dev)
@@ -307,6 +310,18 @@ def run_cuda(args, wl, shape, mask, lens):
         name, val = kv_.split("=")
         ctx.set_option(name, int(val))
     stream = torch.cuda.current_stream()
+
+    if args.prefill_only:
+        if rank == 0:
+            peaks = {}
+            try:
+                peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
+            except Exception:
+                pass
+            print(json.dumps({"prefill_only": True, "layers": L, "options": args.opt,
+                              "prefill": prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, opts=args.opt),
+                              "note": "profiling case, not a benchmark value"}))
+        return
 
     tok0 = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).to(dev)
     tok_a, tok_b = tok0.clone(), tok0.clone()
@@ -504,7 +519,7 @@ def run_cuda(args, wl, shape, mask, lens):
            "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
            "kernel_ms_per_step": cls_ms, "route": route}
     if not args.no_prefill:
-        out["prefill"] = prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks)
+        out["prefill"] = prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, opts=args.opt)
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5, rows=min(B, 32), layers=4)
         out["cpu_baseline"].pop("ms_per_step", None)
@@ -524,6 +539,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-route", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prompt-phase leg (first_prefill on this workload's prompts)")
+    ap.add_argument("--prefill-only", action="store_true",
+                    help="only the prompt-phase leg (for profiler captures with --layers; not a benchmark line)")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (A/B runs)")
     ap.add_argument("--layers", type=int, default=None,
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
