@@ -112,6 +112,51 @@ def test_config3_shape_b256_heterogeneous_masks(w8b):
     _stand_in_case(shape, w, gw, om, lens, mask, list(range(0, B, 32)), 2, 23, "config3")
 
 
+def test_8b_shape_one_call_prefill_short_prompts(w8b):
+    """Llama-3-8B shape (head_dim 128, 4 query heads per KV head, 32 layers): the prompt phase of three short
+    prompts in one first_prefill call, in two chunks (48 + 22 rows), against the oracle's prefill: caches of
+    all layers, first logits, then two routed steps.  (Long prompts at this shape are beyond the host oracle.)"""
+    import torch
+    from paper_2410_12513_b200 import FirstContext
+    w, gw, om = w8b
+    shape, lens, S = fi.LLAMA_8B, [33, 9, 28], 2
+    L, B = shape.n_layers, len(lens)
+    prompts = [fi.tokens(shape, n, 2100, f"prompt{b}") for b, n in enumerate(lens)]
+    caps = [n + S for n in lens]
+    okv = oracle.OracleKV(om.shape, caps)
+    pre = [oracle.prefill(om, okv, b, prompts[b], want_router_in=False) for b in range(B)]
+    gkv = GpuKV(shape, caps, True)
+    ctx = FirstContext(shape, 1, 48, max(caps), gw)
+    logits = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda")
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ctx.prefill(torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda(), cu, gkv.c, logits=logits)
+    assert ctx.device_flags() == 0
+    ref0 = np.stack([np.asarray(pre[b]["logits"]).reshape(-1, shape.vocab)[0] for b in range(B)])
+    got = logits.cpu().numpy()
+    err, agree = logits_check(got, ref0)
+    _account(err, agree, got, ref0, "prefill_8b")
+    assert np.array_equal(gkv.len.cpu().numpy(), okv.len) and np.array_equal(gkv.pos.cpu().numpy(), okv.pos)
+    for l in range(L):
+        for b in range(B):
+            n = lens[b]
+            k1, v1 = gkv.rows_host(l, b)
+            ko, vo = okv.rows(l, b)
+            assert np.abs(k1[:n] - ko[:n]).max() <= 2e-2 * max(1.0, np.abs(ko[:n]).max()), (l, b)
+            assert np.abs(v1[:n] - vo[:n]).max() <= 2e-2 * max(1.0, np.abs(vo[:n]).max()), (l, b)
+    mask = fi.mask_skip_fraction(B, L, 0.1, 0.4, 2101)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = oracle.argmax(ref0)
+    for t in range(S):
+        ref = oracle.decode_step(om, toks, mask, okv)
+        ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits)
+        got = logits.cpu().numpy()
+        err, agree = logits_check(got, ref)
+        _account(err, agree, got, ref, "prefill_8b")
+        toks = oracle.argmax(ref)
+    assert ctx.device_flags() == 0
+    ctx.close()
+
+
 _cfg1 = {}
 
 
