@@ -527,8 +527,9 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             c->pdl_next = false;
         }
         if (ph && ph->router_w) {  // prefill: router l reads the rows entering layer l
-            const int blocks = std::min((B + 7) / 8, c->n_sm * 8);
-            FIRST_LAUNCH(kClsRouterScores, (router_token_scores<float><<<blocks, 256, (size_t)D * sizeof(float), st>>>(
+            // a chunk has at most 256 rows: two warps (tokens) per block spread them over the SMs
+            const int blocks = std::min((B + 1) / 2, c->n_sm * 8);
+            FIRST_LAUNCH(kClsRouterScores, (router_token_scores<float><<<blocks, 64, (size_t)D * sizeof(float), st>>>(
                                                c->x, (int64_t)B, D, ph->router_w + (size_t)l * D,
                                                ph->router_b ? ph->router_b + l : nullptr, ph->mode,
                                                ph->tokscore + (size_t)l * ph->stride + ph->g0)));

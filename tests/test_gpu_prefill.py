@@ -168,3 +168,84 @@ def test_prefill_argument_errors_and_short_slab():
     for l in range(shape.n_layers):
         k1, v1 = guard.rows_host(l, 1)
         assert k1[:3].any() and not k1[3:].any() and not v1[3:].any()
+
+
+def test_prefill_joins_a_running_batch():
+    """Continuous batching with the one-call prompt phase: two sequences are prefilled together and decode;
+    a third then joins (prefilled alone into its own slab of the same cache tensors, routed by its own prompt)
+    and the three decode together.  The join must leave the running sequences' slabs bit-identical, and every
+    sequence must follow the oracle run on that sequence alone."""
+    import torch
+    from paper_2410_12513_b200 import KVCache
+    shape, seed, bf16 = SMALL_GQA, 41, True
+    L = shape.n_layers
+    w = fi.make_weights(shape, seed, bf16)
+    om = oracle_model(shape, w)
+    lens, caps = [37, 52, 20], [48, 64, 32]
+    prompts = [fi.tokens(shape, n, seed, f"prompt{b}") for b, n in enumerate(lens)]
+    okvs = [oracle.OracleKV(om.shape, [caps[b]]) for b in range(3)]
+    pre = [oracle.prefill(om, okvs[b], 0, prompts[b]) for b in range(3)]
+    target = np.array([[1, 0, 1], [1, 1, 0], [0, 1, 1]], np.uint8)
+    # one router set serves all three prompts (as it would in a deployment)
+    routers = np.stack([calibrate_router([pre[b]["router_in"][l] for b in range(3)], target[:, l], 0, l)[0]
+                        for l in range(L)])
+    gkv = GpuKV(shape, caps, bf16)
+    ctx = _ctx(shape, bf16, 16, max(caps), w)
+    rw = to_dev(routers, False)
+    mask = torch.zeros((3, L), dtype=torch.uint8, device="cuda")
+    logits = torch.empty((3, shape.vocab), dtype=torch.float32, device="cuda")
+
+    def sub_kv(rows):
+        r = torch.tensor(rows, device="cuda")
+        return (KVCache(gkv.k, gkv.v, gkv.slab_off[r].contiguous(), gkv.slab_cap[r].contiguous(),
+                        gkv.len[:, r].contiguous(), gkv.pos[r].contiguous()), r)
+
+    def write_back(kvc, r):
+        gkv.len[:, r] = kvc.len
+        gkv.pos[r] = kvc.pos
+
+    def first_logits(b):
+        return np.asarray(pre[b]["logits"]).reshape(-1, shape.vocab)[0]
+
+    def decode(rows, kvc, toks, n):
+        for _ in range(n):
+            ref = np.stack([oracle.decode_step(om, toks[i:i + 1], target[b:b + 1], okvs[b])[0] for i, b in enumerate(rows)])
+            ctx.decode_step(torch.from_numpy(toks).cuda(), kvc, logits[:len(rows)])
+            err, agree = logits_check(logits[:len(rows)].cpu().numpy(), ref)
+            assert err.max() <= 2e-2, err.max()
+            toks = oracle.argmax(ref)
+        assert ctx.device_flags() == 0
+        return toks
+
+    # sequences 0 and 2 arrive first
+    kv02, r02 = sub_kv([0, 2])
+    m02 = torch.zeros((2, L), dtype=torch.uint8, device="cuda")
+    cu = np.array([0, lens[0], lens[0] + lens[2]], np.int32)
+    ctx.prefill(torch.from_numpy(np.concatenate([prompts[0], prompts[2]]).astype(np.int32)).cuda(), cu, kv02, rw,
+                None, 0.5, 0, m02, None, logits[:2])
+    assert np.array_equal(m02.cpu().numpy(), target[[0, 2]])
+    err, _ = logits_check(logits[:2].cpu().numpy(), np.stack([first_logits(0), first_logits(2)]))
+    assert err.max() <= 2e-2
+    ctx.set_mask(m02)
+    toks = decode([0, 2], kv02, oracle.argmax(np.stack([first_logits(0), first_logits(2)])), 2)
+    write_back(kv02, r02)
+
+    # sequence 1 joins: its prompt phase must not touch the other slabs
+    before = {(l, b): gkv.rows_host(l, b) for l in range(L) for b in (0, 2)}
+    kv1, r1 = sub_kv([1])
+    m1 = torch.zeros((1, L), dtype=torch.uint8, device="cuda")
+    ctx.prefill(torch.from_numpy(prompts[1].astype(np.int32)).cuda(), np.array([0, lens[1]], np.int32), kv1, rw, None,
+                0.5, 0, m1, None, logits[:1])
+    write_back(kv1, r1)
+    assert np.array_equal(m1.cpu().numpy(), target[1:2])
+    for (l, b), (k0, v0) in before.items():
+        k1, v1 = gkv.rows_host(l, b)
+        assert np.array_equal(k0, k1) and np.array_equal(v0, v1)
+    tok1 = oracle.argmax(first_logits(1)[None])
+    mask.copy_(torch.from_numpy(target))
+    ctx.set_mask(mask)
+    toks3 = np.array([toks[0], tok1[0], toks[1]], np.int32)
+    decode([0, 1, 2], gkv.c, toks3, 3)
+    want_len = np.stack([okvs[b].len[:, 0] for b in range(3)], 1)
+    assert np.array_equal(gkv.len.cpu().numpy(), want_len)
+    assert gkv.pos.cpu().numpy().tolist() == [int(okvs[b].pos[0]) for b in range(3)]
