@@ -323,6 +323,8 @@ const char *first_kernel_class_name(int32_t k);
  *   "fuse_rope"      0 = a separate kernel rotates q/k and appends the new key/value before attention.
  *                    Default 1: the tuned attention kernel (bfloat16 caches, head_dim 64/128) does both
  *                    itself, from the QKV projection's output.
+ *   "prefill_pair"   0 = in first_prefill every prompt token has attention work items of its own.  Default 1:
+ *                    two consecutive tokens of a sequence share them (up to 4 query heads per KV head).
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
  *                    its epilogue (needs ffn_dim % 64 == 0).

@@ -68,7 +68,13 @@ struct RopeFuse {
 // Scratch: o_part [m][Hq][S_max][HD] (unnormalised), ml_part [m][Hq][S_max] = (max, sum),
 // ticket [m][Hkv] (zero between launches: the merging CTA resets it).
 // Output: out [m][Hq*HD] float32 and/or its bfloat16 hi/lo split (either may be NULL).
-template <int HD, int G>
+//
+// PAIR (prompt processing, where consecutive rows are consecutive tokens of one sequence): a work item may
+// serve two rows at once.  rowinfo[i].y bit 61 = row i also serves row i+1 (same slab, one token more, its key
+// and value already in the slab); bit 60 = row i is served by row i-1 (its CTAs exit).  The second row's query
+// heads take fragment rows G..2G-1 (so 2G <= 8), share every K/V tile with the first row's, and see one token
+// more at the end.  Not combined with RopeFuse.
+template <int HD, int G, bool PAIR = false>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
                                                       const float* q, int64_t cap_total,
@@ -82,7 +88,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     constexpr int kBox = kTile * 128;             // bytes of one 64-token x 64-element box
     constexpr int kStageBytes = 2 * kHalves * kBox;
     constexpr int kKSteps = HD / 16, kNTiles = HD / 8;
-    static_assert(G <= 8, "query heads of a group are the 8 hi rows of the A fragment");
+    constexpr int GR = PAIR ? 2 * G : G;  // fragment rows in use
+    static_assert(GR <= 8, "query heads of a group (of two rows' groups) are the 8 hi rows of the A fragment");
 
     pdl_trigger();
     // Set-up that needs nothing from the previous kernel comes first, so that it overlaps that kernel's tail.
@@ -106,10 +113,13 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
     const longlong2 ri = __ldcg(&rowinfo[i]);
-    const int T = (int)(ri.x & 0xffffffffll);
+    const int T1 = (int)(ri.x & 0xffffffffll);  // tokens row i attends over
     const int brow = (int)(ri.x >> 32);
-    const int64_t slab0 = ri.y & ((1ll << 62) - 1);
-    const bool append = rf.qkv != nullptr && (ri.y >> 62) != 0;
+    const int64_t slab0 = ri.y & ((1ll << 60) - 1);
+    const bool append = !PAIR && rf.qkv != nullptr && ((ri.y >> 62) & 1) != 0;
+    if (PAIR && ((ri.y >> 60) & 1)) return;              // row i-1's work items serve this row
+    const bool two = PAIR && ((ri.y >> 61) & 1);          // this work item also serves row i+1
+    const int T = T1 + (two ? 1 : 0);                     // tokens streamed
     // A row of T tokens is cut into ceil(T / C) chunks of equal length (a multiple of the tile), not
     // into full chunks plus a short remainder: its CTAs then finish together.
     const int n_chunks = (T + C - 1) / C;
@@ -155,7 +165,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     uint32_t qh[kKSteps][2], ql[kKSteps][2];  // A fragments: (k0..k0+1), (k0+8..k0+9) of row g
     const int qkv_stride = (Hq + 2 * (int)gridDim.y) * HD;
     const float2* csr = rf.cs + (size_t)brow * (HD / 2);
-    if (rf.qkv) {
+    const int rows_live = two ? 2 * G : G;                // fragment rows that carry a query head
+    if (!PAIR && rf.qkv) {
         constexpr int kHalf = HD / 2;
         const float* qrow = rf.qkv + (size_t)i * qkv_stride + ((size_t)h * G + (g < G ? g : 0)) * HD;
         auto rot2 = [&](int dd) {  // rotated, scaled q[dd], q[dd+1] (dd even; both on the same side of HD/2)
@@ -177,11 +188,12 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
             split2(v1.x, v1.y, qh[ks][1], ql[ks][1]);
         }
     } else {
-        const float* qrow = q + ((size_t)i * Hq + (size_t)h * G + (g < G ? g : 0)) * HD;
+        const int gq = g < rows_live ? g : 0;
+        const float* qrow = q + ((size_t)(i + gq / G) * Hq + (size_t)h * G + gq % G) * HD;
 #pragma unroll
         for (int ks = 0; ks < kKSteps; ++ks) {
             float2 v0 = make_float2(0.f, 0.f), v1 = v0;
-            if (g < G) {
+            if (g < rows_live) {
                 v0 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 2 * tq);
                 v1 = *reinterpret_cast<const float2*>(qrow + ks * 16 + 8 + 2 * tq);
             }
@@ -203,6 +215,8 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
         const uint32_t sK = base + (uint32_t)s * kStageBytes, sV = sK + kHalves * kBox;
         const int tile_t0 = t_begin + j * kTile;
         const int valid = t_end - tile_t0;  // tokens of this tile that exist (may exceed 64)
+        // the first row of a pair does not see the last token (its successor's)
+        const int lim = valid - ((two && g < G && t_end == T) ? 1 : 0);
         if (valid < kTile) {
             // rows past the end hold someone else's bytes: zero them in V so 0 * garbage stays 0
             uint8_t* vptr = base_ptr + (size_t)s * kStageBytes + kHalves * kBox;
@@ -265,7 +279,7 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int tok = warp * 16 + nt * 8 + 2 * tq + e;
-                const float v = (tok < valid) ? sc[nt][e] + sc[nt][e + 2] : -INFINITY;  // hi + lo parts
+                const float v = (tok < lim) ? sc[nt][e] + sc[nt][e + 2] : -INFINITY;  // hi + lo parts
                 sv[nt * 2 + e] = v;
                 mx = fmaxf(mx, v);
             }
@@ -307,20 +321,21 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
     bar_consumers();
-    float* o_s = reinterpret_cast<float*>(base_ptr);       // [4][G][HD]
-    float* m_s = o_s + 4 * G * HD;                          // [4][G]
-    float* l_s = m_s + 4 * G;                               // [4][G]
-    if (g < G) {
+    float* o_s = reinterpret_cast<float*>(base_ptr);       // [4][GR][HD]
+    float* m_s = o_s + 4 * GR * HD;                         // [4][GR]
+    float* l_s = m_s + 4 * GR;                              // [4][GR]
+    if (g < GR) {
 #pragma unroll
         for (int nt = 0; nt < kNTiles; ++nt) {
             float2 v = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
-            *reinterpret_cast<float2*>(o_s + ((size_t)warp * G + g) * HD + nt * 8 + 2 * tq) = v;
+            *reinterpret_cast<float2*>(o_s + ((size_t)warp * GR + g) * HD + nt * 8 + 2 * tq) = v;
         }
-        if (tq == 0) { m_s[warp * G + g] = m_run; l_s[warp * G + g] = l_run; }
+        if (tq == 0) { m_s[warp * GR + g] = m_run; l_s[warp * GR + g] = l_run; }
     }
     bar_consumers();
     if (!ok || abort_s) return;
-    const size_t hq0 = (size_t)i * Hq + (size_t)h * G;
+    // query head (row-major over [m][Hq]) of fragment row gg: the second row of a pair follows the first
+    auto hq_of = [&](int gg) { return (size_t)(i + gg / G) * Hq + (size_t)h * G + gg % G; };
     auto emit = [&](size_t hq, int d, float y) {
         if (out) out[hq * HD + d] = y;
         if (out_hi) {
@@ -329,24 +344,24 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
             out_lo[hq * HD + d] = __float2bfloat16_rn(y - __bfloat162float(hh));
         }
     };
-    for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
+    for (int e = threadIdx.x; e < rows_live * HD; e += kConsumers) {
         const int gg = e / HD, d = e - gg * HD;
-        const float M = fmaxf(fmaxf(m_s[gg], m_s[G + gg]), fmaxf(m_s[2 * G + gg], m_s[3 * G + gg]));
+        const float M = fmaxf(fmaxf(m_s[gg], m_s[GR + gg]), fmaxf(m_s[2 * GR + gg], m_s[3 * GR + gg]));
         float acc = 0.f, l = 0.f;
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-            const float mw = m_s[w * G + gg];
+            const float mw = m_s[w * GR + gg];
             if (mw > -INFINITY) {
                 const float f = __expf(mw - M);
-                acc += o_s[((size_t)w * G + gg) * HD + d] * f;
-                l += l_s[w * G + gg] * f;
+                acc += o_s[((size_t)w * GR + gg) * HD + d] * f;
+                l += l_s[w * GR + gg] * f;
             }
         }
         if (n_chunks == 1) {
-            emit(hq0 + gg, d, acc / l);  // the whole row in one chunk: done
+            emit(hq_of(gg), d, acc / l);  // the whole row in one chunk: done
         } else {
-            o_part[((hq0 + gg) * S_max + c) * HD + d] = acc;
-            if (d == 0) ml_part[(hq0 + gg) * S_max + c] = make_float2(M, l);
+            o_part[(hq_of(gg) * S_max + c) * HD + d] = acc;
+            if (d == 0) ml_part[hq_of(gg) * S_max + c] = make_float2(M, l);
         }
     }
     if (n_chunks == 1) return;
@@ -363,26 +378,26 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     __threadfence();
     // Merge: (1) all chunk statistics into shared memory at once, (2) one weight per (head, chunk),
     // (3) weighted sums with independent loads.  o_s is free again (everyone passed the barrier).
-    float* w_s = o_s;  // [2][G][64]
-    for (int e = threadIdx.x; e < G * n_chunks; e += kConsumers) {
+    float* w_s = o_s;  // [2][GR][64]
+    for (int e = threadIdx.x; e < rows_live * n_chunks; e += kConsumers) {
         const int gg = e / n_chunks, sidx = e - gg * n_chunks;
-        const float2 ml = __ldcg(&ml_part[(hq0 + gg) * S_max + sidx]);
+        const float2 ml = __ldcg(&ml_part[hq_of(gg) * S_max + sidx]);
         w_s[gg * 64 + sidx] = ml.x;
-        w_s[(G + gg) * 64 + sidx] = ml.y;
+        w_s[(GR + gg) * 64 + sidx] = ml.y;
     }
     bar_consumers();
-    if (threadIdx.x < G) {
+    if (threadIdx.x < rows_live) {
         const int gg = threadIdx.x;
         float M = -INFINITY, den = 0.f;
         for (int sidx = 0; sidx < n_chunks; ++sidx) M = fmaxf(M, w_s[gg * 64 + sidx]);
-        for (int sidx = 0; sidx < n_chunks; ++sidx) den += w_s[(G + gg) * 64 + sidx] * __expf(w_s[gg * 64 + sidx] - M);
+        for (int sidx = 0; sidx < n_chunks; ++sidx) den += w_s[(GR + gg) * 64 + sidx] * __expf(w_s[gg * 64 + sidx] - M);
         const float inv = 1.f / den;
         for (int sidx = 0; sidx < n_chunks; ++sidx) w_s[gg * 64 + sidx] = __expf(w_s[gg * 64 + sidx] - M) * inv;
     }
     bar_consumers();
-    for (int e = threadIdx.x; e < G * HD; e += kConsumers) {
+    for (int e = threadIdx.x; e < rows_live * HD; e += kConsumers) {
         const int gg = e / HD, d = e - gg * HD;
-        const size_t hq = hq0 + gg;
+        const size_t hq = hq_of(gg);
         const float* src = o_part + (hq * S_max) * HD + d;
         const float* wv = w_s + gg * 64;
         float acc = 0.f;

@@ -95,6 +95,7 @@ struct first_ctx {
     int tc_use_lo = 1;
     int fuse_swiglu = 1;
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
+    int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
     int tc_lo_max_rows = 1 << 30;  // the hi/lo activation split is used up to this many active rows, hi alone above
@@ -412,7 +413,7 @@ int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorM
     return FIRST_OK;
 }
 
-template <int HD, int G>
+template <int HD, int G, bool PAIR = false>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
                        const LayerKv* kv, const void* kc, const void* vc, int C, float* out,
                        __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
@@ -425,7 +426,7 @@ int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorM
         rf.k_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(kc));
         rf.v_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(vc));
     }
-    return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
+    return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G, PAIR>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
                     c->rowinfo, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
                     out_hi, out_lo, c->flags, rf);
 }
@@ -434,6 +435,8 @@ template <int HD, int G>
 int attn_mma_set_attr() {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    if constexpr (2 * G <= 8)  // the two-rows-per-work-item form used on prompt chunks
+        CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     return FIRST_OK;
 }
 
@@ -450,7 +453,7 @@ int attn_mma_setup(first_ctx* c) {
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const LayerKv* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
-                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
+                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair = false) {
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -470,6 +473,12 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     int rc;
     if ((rc = kv_map_for(c, kc, kv->cap_total, &tk)) || (rc = kv_map_for(c, vc, kv->cap_total, &tv))) return rc;
     dim3 grid(S, d.n_kv_heads, m);
+#define FIRST_ATTN_PAIR(HD, G)                            \
+    if (pair && d.head_dim == HD && c->group == G)        \
+        return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale);
+    FIRST_ATTN_PAIR(128, 1) FIRST_ATTN_PAIR(128, 2) FIRST_ATTN_PAIR(128, 3) FIRST_ATTN_PAIR(128, 4)
+    FIRST_ATTN_PAIR(64, 1) FIRST_ATTN_PAIR(64, 2) FIRST_ATTN_PAIR(64, 3) FIRST_ATTN_PAIR(64, 4)
+#undef FIRST_ATTN_PAIR
 #define FIRST_ATTN_MMA(HD, G)                 \
     if (d.head_dim == HD && c->group == G)    \
         return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale);
@@ -519,6 +528,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const int norm_threads = std::max(32, std::min(1024, (D / 4 + 31) / 32 * 32));  // one float4 per thread when the row allows
     const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
     const bool fuse_rope = mma_attn && c->fuse_rope;
+    // prompt chunks: consecutive rows are consecutive tokens of a sequence and may share attention work items
+    const bool pair_rows = ph && mma_attn && !fuse_rope && c->prefill_pair && 2 * c->group <= 8;
 
     for (int l = 0; l < L; ++l) {
         if (layer_inputs) {
@@ -564,11 +575,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
                            0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
-                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr)))
+                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0)))
             return rc;
         if (mma_attn) {
             if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], &lkv, len_l, idx, t ? nullptr : c->att, xh, xl,
-                                      fuse_rope, qscale)))
+                                      fuse_rope, qscale, pair_rows)))
                 return rc;
         } else {
             if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], &lkv, len_l, idx))) return rc;
@@ -1050,6 +1061,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "use_pdl")) c->use_pdl = value != 0;
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
     else if (!std::strcmp(name, "fuse_rope")) c->fuse_rope = value != 0;
+    else if (!std::strcmp(name, "prefill_pair")) c->prefill_pair = value != 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;

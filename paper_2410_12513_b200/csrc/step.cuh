@@ -149,12 +149,28 @@ __global__ void __launch_bounds__(64) rope_append(const float* qkv, const int32_
                                                   const int64_t* __restrict__ slab_off,
                                                   const int32_t* __restrict__ slab_cap,
                                                   const int32_t* len_l, uint32_t* __restrict__ flags,
-                                                  longlong2* __restrict__ rowinfo) {
+                                                  longlong2* __restrict__ rowinfo, int pair) {
     pdl_trigger();
     pdl_wait();
     const int i = blockIdx.y, head = blockIdx.x, d = threadIdx.x, b = idx[i];
-    if (rowinfo && head == 0 && d == 0)  // what attention needs to know about this row, in one 16-byte word
-        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]) | ((long long)b << 32), (long long)slab_off[b]);
+    if (rowinfo && head == 0 && d == 0) {  // what attention needs to know about this row, in one 16-byte word
+        long long y = (long long)slab_off[b];
+        if (pair) {
+            // Prompt processing: rows i0, i0+1 that are consecutive tokens of one slab (the first at an even
+            // position, both with room) share attention work items: bit 61 marks the first, bit 60 the second.
+            const int m = gridDim.y;
+            auto is_pair = [&](int i0) {
+                if (i0 < 0 || i0 + 1 >= m) return false;
+                const int b0 = idx[i0], b1 = idx[i0 + 1];
+                const int t0 = len_l[b0];
+                return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == t0 + 1 &&
+                       t0 + 1 < slab_cap[b1] && !(t0 & 1);
+            };
+            if (is_pair(i - 1)) y |= 1ll << 60;
+            else if (is_pair(i)) y |= 1ll << 61;
+        }
+        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]) | ((long long)b << 32), y);
+    }
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
     const float* row = qkv + (size_t)i * (qd + 2 * kvd) + (size_t)head * hd;
