@@ -234,7 +234,10 @@ int tc_ksplit(const first_ctx* c, int tiles, int K, int epi, int m, int slots) {
     if (epi == tc::kEpiStore || epi == tc::kEpiSwiglu) return 1;
     const int kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
     int cap = std::max(1, kblocks / 4);
-    if (c->tc_ksplit_cap) cap = std::min(cap, std::max(1, K / (4 * std::max(std::min(m, 256), 1))));
+    // ... except that idle SMs cost more than the reduction traffic: the bound never goes below the count that
+    // fills one wave of the slots (256 rows: O projection 64 -> 144 work units on 148 SMs)
+    if (c->tc_ksplit_cap)
+        cap = std::min(cap, std::max(std::max(1, K / (4 * std::max(std::min(m, 256), 1))), slots / std::max(tiles, 1)));
     cap = std::min(cap, std::max(1, (2 * slots + tiles - 1) / tiles));  // never more than two waves' worth
     double best_eff = 0.0;
     for (int ks = 1; ks <= cap; ++ks) {
