@@ -532,22 +532,13 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const bool mma_attn = kBf16 && c->tc_ready && (hd == 64 || hd == 128) && c->attn_simple <= 0;
     const bool fuse_rope = mma_attn && c->fuse_rope;
     // prompt chunks: consecutive rows are consecutive tokens of a sequence and may share attention work items
+    const bool route_here = ph && ph->router_w;
     const bool pair_rows = ph && mma_attn && !fuse_rope && c->prefill_pair && 2 * c->group <= 8;
 
     for (int l = 0; l < L; ++l) {
         if (layer_inputs) {
             CU_TRY(cudaMemcpyAsync(layer_inputs + (size_t)l * B * D, c->x, (size_t)B * D * sizeof(float),
                                    cudaMemcpyDeviceToDevice, st));
-            c->pdl_next = false;
-        }
-        if (ph && ph->router_w) {  // prefill: router l reads the rows entering layer l
-            // a chunk has at most 256 rows: two warps (tokens) per block spread them over the SMs
-            const int blocks = std::min((B + 1) / 2, c->n_sm * 8);
-            FIRST_LAUNCH(kClsRouterScores, (router_token_scores<float><<<blocks, 64, (size_t)D * sizeof(float), st>>>(
-                                               c->x, (int64_t)B, D, ph->router_w + (size_t)l * D,
-                                               ph->router_b ? ph->router_b + l : nullptr, ph->mode,
-                                               ph->tokscore + (size_t)l * ph->stride + ph->g0)));
-            if ((rc = check_launch(c))) return rc;
             c->pdl_next = false;
         }
         const int m = c->cnt_h[l];
@@ -567,7 +558,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, static_cast<int32_t*>(nullptr),
                            fuse_rope ? lkv.slab_cap : nullptr, fuse_rope ? c->rowinfo : nullptr,
                            fuse_rope ? static_cast<const int32_t*>(len_l) : nullptr, fuse_rope ? lkv.slab_off : nullptr,
-                           c->flags)))
+                           c->flags,
+                           // prompt chunks (all rows active, idx[i] = i): router l scores the rows it normalises
+                           route_here ? ph->router_w + (size_t)l * D : nullptr,
+                           route_here && ph->router_b ? ph->router_b + l : nullptr, route_here ? ph->mode : 0,
+                           route_here ? ph->tokscore + (size_t)l * ph->stride + ph->g0 : nullptr)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
                               c->qkv, c->qkvd, nullptr, true, zero_qkv)))
@@ -575,7 +570,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         // The tuned attention kernel rotates q itself and appends the new token's key and value (its
         // row facts come from the norm kernel above); the general path has a kernel for that.
         if (!fuse_rope &&
-            (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3(d.n_q_heads + 2 * d.n_kv_heads, m), dim3(hd / 2),
+            (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3((d.n_q_heads + 2 * d.n_kv_heads + 7) / 8, m), dim3(hd / 2, 8),
                            0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
                            lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0)))
@@ -595,7 +590,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             return rc;
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->ffn_norm[l],
-                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, lkv.slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
+                           d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, lkv.slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
+                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
@@ -634,7 +630,8 @@ int logits_tail(first_ctx* c, cudaStream_t st, int B, float* logits, int32_t* ne
         const bool t = tc_for(B);
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, D, c->final_norm,
                            d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
-                           nullptr, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr))))
+                           nullptr, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
+                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
             return rc;
         if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
                               nullptr, false)))

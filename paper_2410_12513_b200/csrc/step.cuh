@@ -61,6 +61,9 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 //             word: x = tokens to attend over (cache length + the new token, at most the slab's
 //             capacity) | batch row << 32;  y = first slab row | (1 << 62 when the new token's key
 //             and value are to be appended).  A full slab raises FIRST_FLAG_KV_FULL.
+//   router:   (prompt processing) the row is also what the layer's router reads: its score
+//             z = router_w . x[b] (+ bias) goes to tok_out[i], as sigmoid(z) in the paper's order
+//             (mean of per-token sigmoids) or as z in the pooled order, like router_token_scores.
 __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32_t* __restrict__ idx, int D,
                                                      const float* __restrict__ gain, float eps, float* __restrict__ out,
                                                      __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
@@ -69,7 +72,10 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
                                                      longlong2* __restrict__ rowinfo,
                                                      const int32_t* len_ro,
                                                      const int64_t* __restrict__ slab_off,
-                                                     uint32_t* __restrict__ flags) {
+                                                     uint32_t* __restrict__ flags,
+                                                     const float* __restrict__ router_w,
+                                                     const float* __restrict__ router_b, int router_mode,
+                                                     float* __restrict__ tok_out) {
     // One pass: the row stays in registers between the sum of squares and the scaling
     // (up to kMaxV float4 per thread; longer rows re-read the tail from L1/L2).
     constexpr int kMaxV = 4;
@@ -85,6 +91,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
     const int b = idx ? idx[i] : i;  // the plan is fixed between first_set_mask calls: no need to wait for it
     pdl_wait();
     __shared__ float red[32];
+    __shared__ float red_r[32];
     if (len_inc && threadIdx.x == 0) {
         const int T = len_inc[b];
         if (T < slab_cap[b]) len_inc[b] = T + 1;
@@ -98,21 +105,34 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
     }
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)b * D);
     float4 r[kMaxV];
-    float ss = 0.f;
+    float ss = 0.f, rd = 0.f;
+    const float4* rw4 = reinterpret_cast<const float4*>(router_w);
 #pragma unroll
     for (int v = 0; v < kMaxV; ++v) {
         const int k = threadIdx.x + v * nt;
         if (k < nv) {
             r[v] = xr[k];
             ss += r[v].x * r[v].x + r[v].y * r[v].y + r[v].z * r[v].z + r[v].w * r[v].w;
+            if (router_w) {
+                const float4 w = __ldg(rw4 + k);
+                rd += r[v].x * w.x + r[v].y * w.y + r[v].z * w.z + r[v].w * w.w;
+            }
         }
     }
     for (int k = threadIdx.x + kMaxV * nt; k < nv; k += nt) {
         const float4 v = xr[k];
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        if (router_w) {
+            const float4 w = __ldg(rw4 + k);
+            rd += v.x * w.x + v.y * w.y + v.z * w.z + v.w * w.w;
+        }
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    if (router_w) {
+        rd = warp_sum(rd);
+        if ((threadIdx.x & 31) == 0) red_r[threadIdx.x >> 5] = rd;
+    }
     if (zero_row) {
         float4* z = reinterpret_cast<float4*>(zero_row + (size_t)i * zero_cols);
         for (int k = threadIdx.x; k < zero_cols / 4; k += nt) z[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -120,6 +140,11 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
     __syncthreads();
     float tot = 0.f;
     for (int w = 0; w < (nt >> 5); ++w) tot += red[w];
+    if (router_w && threadIdx.x == 0) {
+        float z = router_b ? router_b[0] : 0.f;
+        for (int w = 0; w < (nt >> 5); ++w) z += red_r[w];
+        tok_out[i] = (router_mode == FIRST_ROUTER_MEAN_OF_SIGMOID) ? 1.f / (1.f + expf(-z)) : z;
+    }
     const float inv = rsqrtf(tot / (float)D + eps);
     auto emit = [&](int k, const float4& v, const float4& gg) {
         const float y[4] = {v.x * inv * gg.x, v.y * inv * gg.y, v.z * inv * gg.z, v.w * inv * gg.w};
@@ -136,13 +161,13 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
 
 // After the QKV projection: rotate q and k at the sequence's position, scale q by
 // 1/sqrt(hd), write k and v at row len[l][b] of the sequence's slab.
-// qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  grid (Hq+2*Hkv, m): one block of
-// hd/2 threads per (row, head); thread d handles the rotary pair (d, d+hd/2).
+// qkv: [m][(Hq+2Hkv)*hd] float32 (q heads, k heads, v heads).  grid (ceil((Hq+2*Hkv)/8), m), block
+// (hd/2, 8): eight heads of a row per block; thread (d, .) handles the rotary pair (d, d+hd/2) of its head.
 // len is only read here (the FFN-side rmsnorm_rows advances it once attention is done).
 // rowinfo[i] = (tokens to attend over, first slab row) saves the attention CTAs two dependent loads.
 // A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
-__global__ void __launch_bounds__(64) rope_append(const float* qkv, const int32_t* __restrict__ idx,
+__global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32_t* __restrict__ idx,
                                                   int Hq, int Hkv, int hd, const float2* cs,
                                                   float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
                                                   KT* __restrict__ vc, int64_t cap_total,
@@ -152,7 +177,8 @@ __global__ void __launch_bounds__(64) rope_append(const float* qkv, const int32_
                                                   longlong2* __restrict__ rowinfo, int pair) {
     pdl_trigger();
     pdl_wait();
-    const int i = blockIdx.y, head = blockIdx.x, d = threadIdx.x, b = idx[i];
+    const int i = blockIdx.y, head = blockIdx.x * blockDim.y + threadIdx.y, d = threadIdx.x, b = idx[i];
+    if (head >= Hq + 2 * Hkv) return;
     if (rowinfo && head == 0 && d == 0) {  // what attention needs to know about this row, in one 16-byte word
         long long y = (long long)slab_off[b];
         if (pair) {
