@@ -200,9 +200,9 @@ int first_prefill_route_static(int32_t layer, int32_t n_layers, int32_t d_model,
  * Whatever the slabs held before is overwritten from row 0.
  *
  * How it runs: the prompt tokens go through the kernels of first_decode_step in chunks of
- * min(max_batch, 256) tokens, each token a row of its own (its slab is its sequence's slab, its
- * cache length its position), so a context meant for prefill should be created with max_batch
- * of 256 or more.  Weights are streamed once per chunk.  The chunks run without CUDA graphs.
+ * min(max_batch, 256) tokens (option "prefill_rows"), each token a row of its own (its slab is
+ * its sequence's slab, its cache length its position), so a context meant for prefill should
+ * be created with max_batch of 256 or more.  Weights are streamed once per chunk.  The chunks run without CUDA graphs.
  *   tokens        dev int32 [total], total = cu_seqlens[B]
  *   cu_seqlens    HOST int32 [B+1], cu_seqlens[0] = 0, strictly increasing (no empty prompt);
  *                 every prompt at most max_tokens_per_seq tokens, B at most max_batch
@@ -325,6 +325,7 @@ const char *first_kernel_class_name(int32_t k);
  *                    itself, from the QKV projection's output.
  *   "prefill_pair"   0 = in first_prefill every prompt token has attention work items of its own.  Default 1:
  *                    two consecutive tokens of a sequence share them (up to 4 query heads per KV head).
+ *   "prefill_rows"   prompt tokens per chunk of first_prefill, 1..256 (default 256; never more than max_batch)
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
  *                    its epilogue (needs ffn_dim % 64 == 0).
