@@ -17,7 +17,9 @@
  * This library is the decode-time hot path of that: score the routers on prefill hidden
  * states (first_prefill_route), turn the per-sequence masks into per-layer lists of
  * active rows (first_set_mask), and run decode steps in which each layer's kernels see
- * only the rows that keep it (first_decode_step).
+ * only the rows that keep it (first_decode_step).  first_prefill is the step before it:
+ * the whole prompt phase of a ragged batch (caches of all layers, router decisions, first
+ * token) in one call, for callers that have no prefill of their own.
  *
  * General conventions
  *   - Every function returns a status: 0 = FIRST_OK, negative = error; nothing throws.
