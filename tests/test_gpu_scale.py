@@ -157,6 +157,46 @@ def test_8b_shape_one_call_prefill_short_prompts(w8b):
     ctx.close()
 
 
+def test_config2_prompts_one_call_prefill_sampled_against_the_oracle(w8b):
+    """The prompt phase in the configuration bench.py times: 8B shape, config 2's 32 prompts (128-2048 tokens,
+    34.8 k in all), 256-row chunks that span sequence boundaries.  A full oracle prefill is out of reach at this
+    size, so sampled outputs are checked: attention is causal, hence the keys and values of the first two layers at
+    positions 0..n-1 of a sequence depend on its first n tokens only, and a two-layer oracle on that prefix gives
+    them.  Sampled: 40-token prefixes of four sequences spread over the batch and a 300-token prefix (it crosses a
+    chunk boundary).  len/pos are checked for every sequence."""
+    import torch
+    from paper_2410_12513_b200 import FirstContext
+    w, gw, om = w8b
+    shape = fi.LLAMA_8B
+    B, L = 32, shape.n_layers
+    lens = fi.prompt_lengths(B, 128, 2048, 1000)
+    prompts = [fi.tokens(shape, int(n), 2200, f"prompt{b}") for b, n in enumerate(lens)]
+    caps = (lens + 2).astype(np.int32)
+    gkv = GpuKV(shape, caps, True)
+    ctx = FirstContext(shape, 1, 256, int(caps.max()), gw)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    nxt = torch.empty((B,), dtype=torch.int32, device="cuda")
+    ctx.prefill(torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda(), cu, gkv.c, next_tokens=nxt)
+    assert ctx.device_flags() == 0
+    assert np.array_equal(gkv.len.cpu().numpy(), np.broadcast_to(lens.astype(np.int32), (L, B)))
+    assert np.array_equal(gkv.pos.cpu().numpy(), lens.astype(np.int32))
+    assert ((nxt.cpu().numpy() >= 0) & (nxt.cpu().numpy() < shape.vocab)).all()
+    # two-layer oracle on prefixes
+    d2 = shape.asdict()
+    d2["n_layers"] = 2
+    shape2 = fi.ModelShape(**d2)
+    w2 = {k: (v[:2] if isinstance(v, list) else v) for k, v in w.items()}
+    om2 = oracle_model(shape2, w2)
+    for b, n in ((0, 40), (7, 40), (19, 40), (31, 40), (12, min(300, int(lens[12])))):
+        ref = oracle.forward_full(om2, prompts[b][:n], want_kv=True)
+        for l in range(2):
+            k1, v1 = gkv.rows_host(l, b)
+            ko, vo = ref["k"][l], ref["v"][l]
+            assert np.abs(k1[:n] - ko).max() <= 2e-2 * max(1.0, np.abs(ko).max()), (b, l)
+            assert np.abs(v1[:n] - vo).max() <= 2e-2 * max(1.0, np.abs(vo).max()), (b, l)
+    ctx.close()
+
+
 _cfg1 = {}
 
 
