@@ -114,6 +114,18 @@ def test_prefill_bf16_gqa_ragged(max_batch):
     _prefill_case(SMALL_GQA, True, [8, 200, 77, 130, 1], max_batch, 3, 5, 0, 0.6, 2e-2)
 
 
+@pytest.mark.parametrize("hq,hkv,hd", [(4, 4, 64), (4, 2, 128), (6, 2, 64), (8, 1, 64)])
+def test_prefill_bf16_query_head_groupings(hq, hkv, hd):
+    """1, 2, 3 and 8 query heads per KV head: the first three let two consecutive prompt tokens share an
+    attention work item (their query heads fit the spare fragment rows), the last does not."""
+    shape = fi.ModelShape(2, hq * hd, hq, hkv, hd, 512, 1024, 500000.0)
+    _prefill_case(shape, True, [70, 3, 131], 64, 2, 8, 0, 0.6, 2e-2)
+
+
+def test_prefill_bf16_pairing_off_by_option():
+    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"prefill_pair": 0, "prefill_rows": 20})
+
+
 def test_prefill_bf16_general_kernels_by_option():
     _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"attn_simple": 1, "max_gemv_rows": 1024})
 
