@@ -68,6 +68,8 @@ extern "C" {
 #define FIRST_FLAG_BAD_MASK 4u     /* mask byte other than 0 or 1 */
 #define FIRST_FLAG_WAIT_EXPIRED 8u /* a bounded wait inside a kernel gave up */
 #define FIRST_FLAG_EMPTY_SEQ 16u   /* a router call saw a sequence with no tokens */
+#define FIRST_FLAG_BAD_SEQ_TABLE 32u /* a router call saw cu_seqlens entries that are negative, decreasing or
+                                        beyond total_tokens; that sequence's mask byte and score are unwritten */
 
 #define FIRST_ROUTER_MEAN_OF_SIGMOID 0 /* the paper's order: rho = mean_j sigmoid(z_j) */
 #define FIRST_ROUTER_SIGMOID_OF_MEAN 1 /* pooled variant:    rho = sigmoid(mean_j z_j) */
@@ -144,7 +146,10 @@ int first_destroy(first_ctx *ctx);
  *                 at least one token (an empty one sets FIRST_FLAG_EMPTY_SEQ and its mask
  *                 byte and score are left unwritten)
  *   total_tokens  host value of cu_seqlens[B] (sizes the launch); at most
- *                 max_batch*max_tokens_per_seq (the scratch capacity)
+ *                 max_batch*max_tokens_per_seq (the scratch capacity).  The device table is checked
+ *                 against it: a sequence whose rows are negative, run backwards or end beyond
+ *                 total_tokens sets FIRST_FLAG_BAD_SEQ_TABLE, reads nothing and leaves its mask
+ *                 byte and score unwritten
  *   router_w      dev float32 [d_model];  router_b  dev float32 [1] or NULL
  *   mask          dev uint8 [B][n_layers] (only column `layer` is written)
  *   scores        dev float32 [B][n_layers] or NULL
@@ -171,7 +176,7 @@ int first_prefill_route(first_ctx *ctx, int32_t layer, const void *hidden, int32
  *
  * Arguments are those of first_prefill_route, with n_layers and d_model passed directly
  * (d_model a multiple of 8, at most 12288) and
- *   flags   dev uint32 [1] or NULL: receives FIRST_FLAG_EMPTY_SEQ (OR-ed in, never cleared
+ *   flags   dev uint32 [1] or NULL: receives FIRST_FLAG_EMPTY_SEQ / FIRST_FLAG_BAD_SEQ_TABLE (OR-ed in, never cleared
  *           here).  With NULL a word inside the built-in scratch is used; it is reset to
  *           zero at the start of every call and cannot be read back by the caller.
  * Limits and rules:

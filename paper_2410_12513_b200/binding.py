@@ -13,7 +13,7 @@ _lib = None
 
 FIRST_DTYPE_F32, FIRST_DTYPE_BF16 = 0, 1
 MEAN_OF_SIGMOID, SIGMOID_OF_MEAN = 0, 1
-FLAG_KV_FULL, FLAG_BAD_TOKEN, FLAG_BAD_MASK, FLAG_WAIT_EXPIRED, FLAG_EMPTY_SEQ = 1, 2, 4, 8, 16
+FLAG_KV_FULL, FLAG_BAD_TOKEN, FLAG_BAD_MASK, FLAG_WAIT_EXPIRED, FLAG_EMPTY_SEQ, FLAG_BAD_SEQ_TABLE = 1, 2, 4, 8, 16, 32
 
 
 class FirstError(RuntimeError):

@@ -783,7 +783,7 @@ int first_prefill_route(first_ctx* c, int32_t layer, const void* hidden, int32_t
                                                               router_w, router_b, mode, c->tokscore)));
     int rc = check_launch(c);
     if (rc) return rc;
-    FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->tokscore, cu_seqlens, c->d.n_layers, layer, mode, tau, mask, scores,
+    FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->tokscore, cu_seqlens, total_tokens, c->d.n_layers, layer, mode, tau, mask, scores,
                                        c->flags)));
     return check_launch(c);
 }
@@ -974,7 +974,7 @@ int first_prefill(first_ctx* c, const int32_t* tokens, const int32_t* cu_seqlens
     }
     if (router_w)
         for (int l = 0; l < L; ++l) {
-            FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->pf_score + (size_t)l * total, c->pf_cu, L, l,
+            FIRST_LAUNCH(kClsRouterFinalize, (router_finalize<<<B, 256, 0, st>>>(c->pf_score + (size_t)l * total, c->pf_cu, total, L, l,
                                                                                  mode, tau, mask, scores, c->flags)));
             if ((rc = check_launch(c))) return rc;
         }

@@ -85,7 +85,7 @@ extern "C" int first_prefill_route_static(int32_t layer, int32_t n_layers, int32
         router_token_scores<float><<<blocks, 256, smem, st>>>(static_cast<const float*>(hidden), total_tokens, d_model,
                                                               router_w, router_b, mode, s->tok);
     if (cudaGetLastError() != cudaSuccess) return FIRST_E_CUDA;
-    router_finalize<<<B, 256, 0, st>>>(s->tok, cu_seqlens, n_layers, layer, mode, tau, mask, scores, fl);
+    router_finalize<<<B, 256, 0, st>>>(s->tok, cu_seqlens, total_tokens, n_layers, layer, mode, tau, mask, scores, fl);
     if (cudaGetLastError() != cudaSuccess) return FIRST_E_CUDA;
     return FIRST_OK;
 }

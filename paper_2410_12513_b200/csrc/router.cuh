@@ -37,13 +37,20 @@ __global__ void __launch_bounds__(256) router_token_scores(const HT* __restrict_
 
 // Pass 2: one block per sequence; float64 mean in a fixed order (strided partial sums
 // then a fixed tree), sigmoid for mode 1, threshold with ">=".
+// The sequence table comes from the caller: a row range that leaves [0, n_tokens] (the token
+// scores pass 1 wrote), or runs backwards, is never followed -- the block raises
+// FIRST_FLAG_BAD_SEQ_TABLE and writes nothing; an empty range raises FIRST_FLAG_EMPTY_SEQ.
 static __global__ void __launch_bounds__(256) router_finalize(const float* __restrict__ tok, const int32_t* __restrict__ cu,
-                                                       int L, int layer, int mode, float tau,
+                                                       int64_t n_tokens, int L, int layer, int mode, float tau,
                                                        uint8_t* __restrict__ mask, float* __restrict__ scores,
                                                        uint32_t* __restrict__ flags) {
     __shared__ double part[256];
     const int b = blockIdx.x;
     const int lo = cu[b], hi = cu[b + 1];
+    if (lo < 0 || hi < lo || (int64_t)hi > n_tokens) {  // uniform over the block
+        if (threadIdx.x == 0) atomicOr(flags, FIRST_FLAG_BAD_SEQ_TABLE);
+        return;
+    }
     double s = 0.0;
     for (int j = lo + threadIdx.x; j < hi; j += 256) s += (double)tok[j];
     part[threadIdx.x] = s;
@@ -53,7 +60,7 @@ static __global__ void __launch_bounds__(256) router_finalize(const float* __res
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        if (hi <= lo) {
+        if (hi == lo) {
             atomicOr(flags, FIRST_FLAG_EMPTY_SEQ);
             return;
         }

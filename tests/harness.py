@@ -119,17 +119,37 @@ def synthetic_caches(shape, lens, caps, seed, bf16, layers=None, with_gpu=True):
 
 
 # ------------------------------------------------------------------ router calibration
-def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3):
+def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3, tight=False):
     """Router weights w[D] (no bias) that realise `target_keep` on the given per-sequence hidden
     states with every oracle score at least `margin` away from tau.  Least-norm solve on the
-    pooled means (B <= D), scaled up until the oracle's own scores clear the margin."""
+    pooled means (B <= D), scaled up until the oracle's own scores clear the margin.
+    tight=True: scaled so that the score nearest to tau lies in [margin, 2*margin] -- the stated
+    margin itself, not a comfortable multiple of it."""
     B = len(hiddens)
     pooled = np.stack([h.astype(np.float64).mean(0) for h in hiddens])  # [B][D]
     t = np.where(np.asarray(target_keep) > 0, 1.0, -1.0)
+    pinv = np.linalg.pinv(pooled)
+
+    # tight: the sequences' distances from tau are spread over [0.7, 1.3] x the middle one
+    spread = np.random.default_rng(seed).permutation(np.linspace(0.7, 1.3, B)) if tight else np.ones(B)
+
+    def scores(c):
+        w = (pinv @ (c * t * spread)).astype(np.float32)
+        rho = np.array([oracle.route(h, w, None, tau, mode)[0] for h in hiddens])
+        return w, rho
+
+    if tight:
+        c = 6.0 * margin  # sigmoid'(0) = 1/4: |rho - 1/2| ~ c/4 = 1.5 margin for the middle sequence
+        for _ in range(40):
+            w, rho = scores(c)
+            gap = np.abs(rho - tau).min()
+            if ((rho >= tau) == (t > 0)).all() and margin <= gap <= 2.0 * margin:
+                return w, rho
+            c *= (1.06 * margin / gap) if gap > 0 else 2.0  # aim the nearest score just outside the margin
+        raise AssertionError("tight router calibration failed")
     c = 0.25
     for _ in range(12):
-        w = (np.linalg.pinv(pooled) @ (c * t)).astype(np.float32)
-        rho = np.array([oracle.route(h, w, None, tau, mode)[0] for h in hiddens])
+        w, rho = scores(c)
         keep = rho >= tau
         if (keep == (t > 0)).all() and np.abs(rho - tau).min() >= margin:
             return w, rho

@@ -50,6 +50,85 @@ def test_router_masks_bit_exact(hidden_bf16, mode):
     assert np.abs(scores.cpu().numpy() - want_rho).max() < 1e-5
 
 
+@pytest.mark.parametrize("hidden_bf16", [False, True])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_router_masks_bit_exact_at_the_stated_margin(hidden_bf16, mode):
+    """Scores as close to tau as the stated margin allows: the router weights are scaled so that the
+    nearest oracle score sits between 1e-3 and 2e-3 from tau (the others up to 2.2e-3).  Identical
+    hidden states on both sides; both router entry points; sequence lengths 1 .. 1111."""
+    import torch
+    from paper_2410_12513_b200 import first_prefill_route_static
+    D, L = 512, 4
+    shape = fi.ModelShape(L, D, 4, 4, 128, 1024, 64)
+    ctx = _ctx(shape, False, 16, 1200, fi.make_weights(shape, 1, False))
+    lens = [1, 7, 300, 33, 1111, 64, 2, 257, 1024, 5]
+    B = len(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    mask = torch.full((B, L), 9, dtype=torch.uint8, device="cuda")
+    mask_s = mask.clone()
+    scores = torch.zeros((B, L), dtype=torch.float32, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    want_mask = np.zeros((B, L), np.uint8)
+    want_rho = np.zeros((B, L))
+    for l in range(L):
+        hid = fi.normal((int(cu[-1]), D), 1.0, 17, f"hid{l}", hidden_bf16)
+        hid_f = widen(hid)
+        hs = [hid_f[cu[b]:cu[b + 1]] for b in range(B)]
+        target = fi.mask_bernoulli(B, 3, 0.5, 200 + l)[:, 1]
+        tau = 0.5 if l < 3 else 0.4
+        rw, _ = calibrate_router(hs, target, mode, l, tau=tau, tight=True)
+        want_rho[:, l], want_mask[:, l] = oracle.route_batch(hid_f, cu, rw, None, tau, mode)
+        gap = np.abs(want_rho[:, l] - tau)
+        assert 1e-3 <= gap.min() <= 2e-3 and gap.max() <= 2.5e-3, gap
+        assert np.array_equal(want_mask[:, l], target)
+        args = (to_dev(hid, hidden_bf16), torch.from_numpy(cu).cuda(), to_dev(rw, False), None, tau, mode)
+        ctx.prefill_route(l, *args, mask, scores)
+        first_prefill_route_static(l, L, *args, mask_s, None, flags)
+    assert ctx.device_flags() == 0 and int(flags.item()) == 0
+    assert np.array_equal(mask.cpu().numpy(), want_mask)
+    assert np.array_equal(mask_s.cpu().numpy(), want_mask)
+    # the device scores are a float32 rounding of the float64 mean: far inside the margin
+    assert np.abs(scores.cpu().numpy() - want_rho).max() < 2e-6
+
+
+def test_router_sequence_table_is_checked_against_total_tokens():
+    """A cu_seqlens whose entries leave [0, total_tokens] or run backwards is never followed: the
+    sequence is flagged, nothing of it is read, its mask byte and score stay as they were."""
+    import torch
+    from paper_2410_12513_b200 import first_prefill_route_static
+    shape = fi.ModelShape(2, 64, 2, 2, 32, 64, 32)
+    ctx = _ctx(shape, False, 4, 64, fi.make_weights(shape, 1, False))
+    hid_h = fi.normal((10, 64), 1.0, 1, "h")
+    hid = to_dev(hid_h, False)
+    rw_h = fi.normal((64,), 0.1, 1, "rw")
+    rw = to_dev(rw_h, False)
+    _, want = oracle.route_batch(hid_h, np.array([0, 4, 10]), rw_h, None, 0.5, 0)
+    for bad in ([0, 4, 11], [0, 12, 10], [-1, 4, 10], [0, 4, 2**31 - 1]):
+        cu = torch.tensor(bad, dtype=torch.int32, device="cuda")
+        for static in (False, True):
+            mask = torch.full((2, 2), 7, dtype=torch.uint8, device="cuda")
+            sc = torch.full((2, 2), -3.0, dtype=torch.float32, device="cuda")
+            if static:
+                fl = torch.zeros(1, dtype=torch.int32, device="cuda")
+                first_prefill_route_static(1, 2, hid, cu, rw, None, 0.5, 0, mask, sc, fl)
+                torch.cuda.synchronize()
+                got_flags = int(fl.item())
+            else:
+                ctx.prefill_route(1, hid, cu, rw, None, 0.5, 0, mask, sc)
+                got_flags = ctx.device_flags()
+            assert got_flags == 32, (bad, static, got_flags)
+            m, s_ = mask.cpu().numpy(), sc.cpu().numpy()
+            good = [b for b in range(2) if 0 <= bad[b] <= bad[b + 1] <= 10]
+            for b in range(2):
+                if b in good:
+                    assert m[b, 1] in (0, 1) and s_[b, 1] != -3.0
+                    if bad[b:b + 2] == [0, 4]:
+                        assert m[b, 1] == want[0]
+                else:
+                    assert m[b, 1] == 7 and s_[b, 1] == -3.0
+            assert (m[:, 0] == 7).all()
+
+
 def test_router_tie_keeps_and_empty_sequence_flag():
     import torch
     shape = fi.ModelShape(2, 64, 2, 2, 32, 64, 32)
@@ -120,7 +199,8 @@ def _run_decode_case(shape, bf16, lens, mask, steps, seed, rel_tol, options=None
         err, agree = logits_check(got, ref)
         errs.append(err)
         agrees.append(agree)
-        assert np.array_equal(nxt.cpu().numpy(), got.argmax(-1).astype(np.int32))  # lowest index of the max
+        assert np.array_equal(nxt.cpu().numpy(), oracle.argmax(got))  # the oracle's greedy rule on the same logits
+        assert np.array_equal(nxt.cpu().numpy(), got.argmax(-1).astype(np.int32))
         toks = oracle.argmax(ref)  # teacher forcing with the oracle's tokens
     errs, agrees = np.stack(errs), np.stack(agrees)
     assert errs.max() <= rel_tol, errs.max()
@@ -185,6 +265,37 @@ def test_decode_bf16_gemv_path_and_general_attention_by_option():
     _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"max_gemv_rows": 8, "attn_simple": 1})
     _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"fuse_swiglu": 0, "use_pdl": 0, "use_graph": 0})
     _run_decode_case(shape, True, lens, mask, 2, 26, 2e-2, options={"fuse_rope": 0})
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_greedy_token_on_exact_ties_is_the_lowest_index(bf16):
+    """lm_head rows v and v + V/2 are the same vector, so every logit occurs (at least) twice, exactly:
+    the greedy token must be the lower index, on the device as in the oracle."""
+    import torch
+    shape = fi.ModelShape(2, 256, 4, 2, 64, 512, 1000, 10000.0)
+    B, V = 6, shape.vocab
+    w = fi.make_weights(shape, 31, bf16)
+    w["lm_head"][V // 2:] = w["lm_head"][:V // 2]
+    om = oracle_model(shape, w)
+    lens = fi.prompt_lengths(B, 1, 40, 31)
+    okv, gkv = synthetic_caches(shape, lens, [int(n) + 2 for n in lens], 31, bf16)
+    ctx = _ctx(shape, bf16, B, int(max(lens)) + 2, w)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.7, 32)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = fi.tokens(shape, B, 31, "first")
+    logits = torch.empty((B, V), dtype=torch.float32, device="cuda")
+    nxt = torch.empty((B,), dtype=torch.int32, device="cuda")
+    nxt_only = torch.empty((B,), dtype=torch.int32, device="cuda")
+    ref = oracle.decode_step(om, toks, mask, okv)
+    ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits, nxt)
+    got = logits.cpu().numpy()
+    assert np.array_equal(ref[:, :V // 2], ref[:, V // 2:]) and np.array_equal(got[:, :V // 2], got[:, V // 2:])
+    want = oracle.argmax(ref)
+    assert (want < V // 2).all()
+    assert np.array_equal(nxt.cpu().numpy(), oracle.argmax(got)) and (nxt.cpu().numpy() < V // 2).all()
+    if not bf16:
+        assert np.array_equal(nxt.cpu().numpy(), want)
+    assert ctx.device_flags() == 0
 
 
 def test_all_skip_and_all_keep_masks():

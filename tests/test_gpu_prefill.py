@@ -23,7 +23,7 @@ def _ctx(shape, bf16, max_batch, max_tokens, w):
     return FirstContext(shape, BF16 if bf16 else F32, max_batch, max_tokens, gpu_weights(w))
 
 
-def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_tol, options=None):
+def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_tol, options=None, tight=False):
     """Oracle prefill per sequence -> routers calibrated on its layer inputs -> one first_prefill
     call on the GPU -> everything it leaves behind compared -> `steps` routed decode steps."""
     import torch
@@ -37,10 +37,12 @@ def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_t
     target = fi.mask_bernoulli(B, L, keep_p, seed + 7)
     routers, rho = [], []
     for l in range(L):
-        rw, r = calibrate_router([pre[b]["router_in"][l] for b in range(B)], target[:, l], mode, l)
+        rw, r = calibrate_router([pre[b]["router_in"][l] for b in range(B)], target[:, l], mode, l, tight=tight)
         routers.append(rw)
         rho.append(r)
     rho = np.stack(rho, 1)  # [B][L]
+    if tight:
+        assert 1e-3 <= np.abs(rho - 0.5).min() <= 2e-3
 
     gkv = GpuKV(shape, caps, bf16)
     ctx = _ctx(shape, bf16, max_batch, max(caps), w)
@@ -98,6 +100,13 @@ def test_prefill_config0_chunks_cross_sequence_boundaries():
     """Tiny fp32 decoder, batch 2, prompts of 32 tokens (config 0), pooled-sigmoid routers; chunks of
     24 rows: 24 + 24 + 16, the second one holding the end of sequence 0 and the start of sequence 1."""
     _prefill_case(fi.TINY, False, [32, 32], 24, 4, 0, 1, 0.6, 1e-4)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_prefill_f32_router_masks_at_the_stated_margin(mode):
+    """float32 model, routers scaled so that the nearest oracle score is 1e-3 .. 2e-3 from tau: the hidden
+    states are the device's own float32 prefill here (not shared bytes), and the masks are still bit-exact."""
+    _prefill_case(fi.TINY, False, [32, 32, 7, 1, 50], 24, 2, 40 + mode, mode, 0.6, 1e-4, tight=True)
 
 
 @pytest.mark.parametrize("max_batch", [5, 64, 300])

@@ -170,8 +170,11 @@ def test_skipped_layer_is_identity_and_leaves_cache_untouched(tiny):
         kv = oracle.OracleKV(model.shape, [n + 4] * B)
         for b in range(B):
             oracle.prefill(model, kv, b, prompts[b])
-        for l in range(s.n_layers):  # poison the unused tail so a stray write shows
-            kv.k[l][:] += 0
+        for l in range(s.n_layers):  # a recognisable non-zero fill beyond each prompt, so a stray write shows
+            for b in range(B):
+                kr, vr = kv.rows(l, b)
+                kr[n:] = 777.0 + l
+                vr[n:] = -777.0 - l
         before = [(k.copy(), v.copy()) for k, v in zip(kv.k, kv.v)]
         tok = np.array([5, 6, 7], np.int32)
         out = []
@@ -247,6 +250,38 @@ def test_batch_permutation_and_single_row_equivalence(tiny):
     assert np.array_equal(run(perm), base[perm])
     for b in range(B):
         assert np.array_equal(run([b])[0], base[b])
+
+
+# ---------------------------------------------------------------- greedy rule (lowest index among equal maxima)
+def test_argmax_takes_the_lowest_index_among_equal_maxima():
+    # hand cases: the expected index is written out, not computed
+    cases = [
+        ([1.0, 3.0, 3.0, 2.0], 1),                       # tie between 1 and 2 -> 1
+        ([5.0, 5.0, 5.0], 0),                            # all equal -> 0
+        ([0.0, -1.0, 2.5], 2),                           # maximum at the last index
+        ([-np.inf, -np.inf, -3.0, -np.inf], 2),          # -inf entries never win over a finite value
+        ([-np.inf, -np.inf], 0),                         # all -inf: still the lowest index
+        ([-0.0, 0.0], 0),                                # signed zeros compare equal
+        ([7.0], 0),
+        ([-2.0, -1.0, -1.0, -3.0, -1.0], 1),
+    ]
+    for row, want in cases:
+        assert oracle.argmax(np.array([row], np.float32)).tolist() == [want], row
+    # a tie planted far apart in a long row, and at the two ends
+    v = np.full(128256, -1.0, np.float32)
+    v[[100000, 17, 128255]] = 4.0
+    assert oracle.argmax(v[None])[0] == 17
+    v[:] = 0.0
+    v[128255] = 1e-30
+    assert oracle.argmax(v[None])[0] == 128255
+    # random rows without and with many ties: numpy's argmax has the same first-occurrence rule
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal((64, 1003)).astype(np.float32)
+    assert np.array_equal(oracle.argmax(a), a.argmax(-1))
+    q = rng.integers(0, 4, (64, 1003)).astype(np.float32)
+    assert np.array_equal(oracle.argmax(q), q.argmax(-1))
+    # a mistake of the ">=" kind would return the LAST maximum: make sure that is told apart
+    assert oracle.argmax(q)[0] != len(q[0]) - 1 - q[0][::-1].argmax()
 
 
 def test_plan_lists_active_rows_in_order():

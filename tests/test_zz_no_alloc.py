@@ -6,7 +6,9 @@ latency path that cannot afford cudaMalloc's device-wide synchronisation).  It k
 scratch in an array built into the library, shared by every call on the device and never
 cleared between calls.  The test therefore makes two calls in a row -- a long batch, then a
 shorter one with different data, so the second runs over the first call's leftovers -- and
-checks both against first_prefill_route: masks bit for bit, scores to float32 rounding.
+checks both against the host oracle (masks bit for bit, scores to float32 rounding) and against
+first_prefill_route.  It also checks the property the entry point exists for: the device's free
+memory is the same before and after a call.
 This file sorts last on purpose: a run that stops at the first failure has by then run
 every other test.
 """
@@ -14,7 +16,8 @@ import numpy as np
 import pytest
 
 import first_inputs as fi
-from harness import gpu_weights, to_dev
+import oracle
+from harness import gpu_weights, to_dev, widen
 
 pytestmark = pytest.mark.gpu
 
@@ -32,13 +35,21 @@ def _both(ctx, L, layer, hid, cu, rw, bias, mode):
     m_new, s_new = m_ref.clone(), s_ref.clone()
     ctx.prefill_route(layer, hid_t, cu_t, rw_t, b_t, 0.5, mode, m_ref, s_ref)
     flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
     first_prefill_route_static(layer, L, hid_t, cu_t, rw_t, b_t, 0.5, mode, m_new, s_new, flags)
     torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
     assert ctx.device_flags() == 0 and int(flags.item()) == 0
+    # against the host oracle on the same bytes
+    rho, keep = oracle.route_batch(widen(hid), cu, rw, bias, 0.5, mode)
+    assert np.abs(rho - 0.5).min() >= 1e-3  # (inputs chosen away from the threshold)
+    assert np.array_equal(m_new[:, layer].cpu().numpy(), keep)
+    assert np.abs(s_new[:, layer].cpu().numpy() - rho).max() <= 2e-6
+    # and against the entry point that takes its scratch from a context
     assert np.array_equal(m_new.cpu().numpy(), m_ref.cpu().numpy())
-    assert set(np.unique(m_new[:, layer].cpu().numpy())) <= {0, 1}
     assert np.abs(s_new.cpu().numpy() - s_ref.cpu().numpy()).max() <= 1e-6
-    return m_new[:, layer].cpu().numpy()
+    return m_new[:, layer].cpu().numpy(), free0, free1
 
 
 def test_static_router_matches_context_router_on_two_calls_in_a_row():
@@ -52,13 +63,15 @@ def test_static_router_matches_context_router_on_two_calls_in_a_row():
     cu1 = np.concatenate([[0], np.cumsum(lens1)]).astype(np.int32)
     hid1 = fi.normal((int(cu1[-1]), D), 1.0, 11, "hid1", True)
     rw1 = fi.normal((D,), 0.05, 11, "rw1")
-    k1 = _both(ctx, L, 1, hid1, cu1, rw1, None, 0)
-    # call 2: shorter batch, float32 hidden states, pooled order, with a bias: runs over call 1's leftovers
+    k1, _, _ = _both(ctx, L, 1, hid1, cu1, rw1, None, 0)
+    # call 2: shorter batch, float32 hidden states, pooled order, with a bias: runs over call 1's leftovers.
+    # By now the array's address has been looked up, so this call must leave the device's free memory as it was.
     lens2 = np.array([5, 40, 9], np.int32)
     cu2 = np.concatenate([[0], np.cumsum(lens2)]).astype(np.int32)
     hid2 = fi.normal((int(cu2[-1]), D), 1.0, 12, "hid2", False)
     rw2 = fi.normal((D,), 0.05, 12, "rw2")
-    k2 = _both(ctx, L, 2, hid2, cu2, rw2, 0.01, 1)
+    k2, free0, free1 = _both(ctx, L, 2, hid2, cu2, rw2, 0.01, 1)
+    assert free1 == free0, (free0, free1)
     assert len(k1) == 6 and len(k2) == 3
     # an empty sequence is reported through the caller's flag word and its outputs are left alone
     cu3 = torch.tensor([0, 0, 5], dtype=torch.int32, device="cuda")
@@ -67,6 +80,14 @@ def test_static_router_matches_context_router_on_two_calls_in_a_row():
     first_prefill_route_static(0, L, to_dev(hid2[:5], False), cu3, to_dev(rw2, False), None, 0.5, 0, m, None, flags)
     torch.cuda.synchronize()
     assert int(flags.item()) == 16 and m[:, 0].cpu().numpy().tolist() == [9, m[1, 0].item()] and m[1, 0].item() in (0, 1)
+    # without a flag word of the caller's the built-in one is used: the call succeeds, the empty sequence's
+    # outputs stay as they were and the other sequence gets what the oracle gives
+    m2 = torch.full((2, L), 9, dtype=torch.uint8, device="cuda")
+    first_prefill_route_static(0, L, to_dev(hid2[:5], False), cu3, to_dev(rw2, False), None, 0.5, 0, m2, None, None)
+    torch.cuda.synchronize()
+    _, keep5 = oracle.route_batch(hid2[:5], np.array([0, 5]), rw2, None, 0.5, 0)
+    assert m2[:, 0].cpu().numpy().tolist() == [9, int(keep5[0])]
+    assert m[1, 0].item() == int(keep5[0])
     # sizes beyond the built-in scratch are refused before anything runs
     too_many = 1048576 + 1
     with pytest.raises(FirstError) as e:
