@@ -2,7 +2,8 @@
 """Benchmark of the router-selective decode step (decode tokens/s and step latency at the
 Llama-3-8B shape, with the achieved fraction of the HBM roofline).
 
-    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library (N > 1: N independent replicas,
+                                                             # started here, one process per GPU, or by torchrun)
     python bench.py --impl reference --steps K --warmup W    # the host oracle, bounded sample
 
 One step = one routed decode step of the whole batch (embedding, every layer for the rows
@@ -94,6 +95,14 @@ def job_tokens_per_s(world, batch_per_rank, steps, ms_max):
     return world * batch_per_rank * steps / (ms_max / 1e3)
 
 
+def physical_gpu_index(local):
+    """nvidia-smi's index of CUDA device `local` of this process (CUDA_VISIBLE_DEVICES may renumber)."""
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")
+    if local < len(vis) and vis[local].strip().isdigit():
+        return int(vis[local])
+    return local
+
+
 class ClockSampler:
     """nvidia-smi sampled every 200 ms while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -149,9 +158,8 @@ class OracleSample:
     (row, layer) count."""
 
     def __init__(self, shape, mask, lens, seed, rows=4, layers=2):
-        sys.path.insert(0, str(ROOT / "tests"))
         import oracle
-        from harness import oracle_model, synthetic_caches
+        from oracle.workload import oracle_model, stand_in_cache
         self.oracle = oracle
         self.B, self.L = mask.shape
         self.rows, self.layers = min(rows, self.B), layers
@@ -162,7 +170,7 @@ class OracleSample:
         sel = np.linspace(0, self.B - 1, self.rows).astype(int)
         l_sel = [int(lens[b]) for b in sel]
         self.caps = [n + 2 for n in l_sel]
-        self.okv, _ = synthetic_caches(sub, l_sel, self.caps, seed, True, with_gpu=False)
+        self.okv = stand_in_cache(sub, l_sel, self.caps, seed, True)
         self.len0, self.pos0 = self.okv.len.copy(), self.okv.pos.copy()
         self.toks = fi.tokens(sub, self.rows, seed, "oracle_tokens")
 
@@ -259,134 +267,297 @@ def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks,
             "note": "prompt tokens as rows of the decode-step kernels, 256 per chunk; weights streamed once per chunk"}
 
 
-# ----------------------------------------------------------------------------- CUDA arm
-def run_cuda(args, wl, shape, mask, lens):
+# ----------------------------------------------------------------------------- replicas (N > 1)
+def init_replica():
+    """(rank, world, local device index, dist module or None, device for the max-over-ranks tensor).
+    Sequences are independent, so N GPUs run N independent replicas: the only communication is the
+    barrier around the timed region and the max over ranks of the device time (NCCL under torchrun,
+    gloo when bench.py starts the replicas itself)."""
     import torch
-    from paper_2410_12513_b200 import FirstContext, KVCache
-
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
+    if world == 1:
+        return rank, world, local, None, None
+    import torch.distributed as dist
+    backend = os.environ.get("FIRST_BENCH_BACKEND", "nccl")
+    if backend == "nccl":
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dev = torch.device("cuda", local)
-    B, L, K, W = mask.shape[0], shape.n_layers, args.steps, args.warmup
-    g = torch.Generator(device=dev)
-    g.manual_seed(1234 + rank)
+        return rank, world, local, dist, torch.device("cuda", local)
+    dist.init_process_group("gloo")
+    return rank, world, local, dist, torch.device("cpu")
 
+
+def free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_replicas(n, argv, script=None, backend="gloo", timeout=3600):
+    """Start n copies of `script argv` (default: this file), replica i on GPU i alone (CUDA_VISIBLE_DEVICES=i,
+    LOCAL_RANK 0), joined by a 127.0.0.1 rendezvous.  Rank 0's standard output is passed through; the return
+    value is the largest exit code."""
+    script = [str(Path(__file__).resolve())] if script is None else list(script)
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), WORLD_SIZE=str(n), LOCAL_RANK="0", LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), CUDA_VISIBLE_DEVICES=str(r),
+                   FIRST_BENCH_BACKEND=backend)
+        procs.append(subprocess.Popen([sys.executable, *script, *argv], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    t_end = time.time() + timeout
+    for pr in procs:
+        try:
+            rc = max(rc, abs(pr.wait(timeout=max(1.0, t_end - time.time()))))
+        except subprocess.TimeoutExpired:
+            pr.kill()  # this replica's own process, by handle
+            rc = max(rc, 124)
+    return rc
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def make_weights_dev(torch, s, dev, g):
     def rnd(shp, std):
         t = torch.empty(shp, dtype=torch.bfloat16, device=dev)
         t.normal_(0.0, std, generator=g)
         return t
 
-    s = shape
-    weights = {"embed": rnd((s.vocab, s.d_model), 0.02), "lm_head": rnd((s.vocab, s.d_model), 0.02),
-               "final_norm": torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g)}
-    for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
-        weights[k] = []
-    for l in range(L):
-        weights["attn_norm"].append(torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g))
-        weights["ffn_norm"].append(torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g))
-        weights["wqkv"].append(rnd((s.q_dim + 2 * s.kv_dim, s.d_model), 0.02))
-        weights["wo"].append(rnd((s.d_model, s.q_dim), 0.02))
-        weights["w_gate_up"].append(rnd((2 * s.ffn_dim, s.d_model), 0.02))
-        weights["w_down"].append(rnd((s.d_model, s.ffn_dim), 0.02))
+    def gain():
+        return torch.ones(s.d_model, device=dev) + 0.02 * torch.randn(s.d_model, device=dev, generator=g)
 
-    phase_steps = W + K
-    caps = (lens + phase_steps + 1).astype(np.int32)
-    off = np.concatenate([[0], np.cumsum(caps[:-1], dtype=np.int64)]).astype(np.int64)
-    tot = int(caps.sum())
-    kk = [rnd((s.n_kv_heads, tot, s.head_dim), 1.0) for _ in range(L)]
-    vv = [rnd((s.n_kv_heads, tot, s.head_dim), 1.0) for _ in range(L)]
-    len0 = torch.from_numpy(np.broadcast_to(lens.astype(np.int32), (L, B)).copy()).to(dev)
-    pos0 = torch.from_numpy(lens.astype(np.int32)).to(dev)
-    len_t, pos_t = len0.clone(), pos0.clone()
-    kv = KVCache(kk, vv, torch.from_numpy(off).to(dev), torch.from_numpy(caps).to(dev), len_t, pos_t)
-    ctx = FirstContext(shape, 1, B, int(caps.max()), weights)
-    for kv_ in args.opt:
-        name, val = kv_.split("=")
-        ctx.set_option(name, int(val))
-    stream = torch.cuda.current_stream()
+    w = {"embed": rnd((s.vocab, s.d_model), 0.02), "lm_head": rnd((s.vocab, s.d_model), 0.02), "final_norm": gain()}
+    for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
+        w[k] = []
+    for _ in range(s.n_layers):
+        w["attn_norm"].append(gain())
+        w["ffn_norm"].append(gain())
+        w["wqkv"].append(rnd((s.q_dim + 2 * s.kv_dim, s.d_model), 0.02))
+        w["wo"].append(rnd((s.d_model, s.q_dim), 0.02))
+        w["w_gate_up"].append(rnd((2 * s.ffn_dim, s.d_model), 0.02))
+        w["w_down"].append(rnd((s.d_model, s.ffn_dim), 0.02))
+    return w
+
+
+class Job:
+    """One workload resident on one GPU: weights, stand-in caches of `lens` tokens with room for `room`
+    more, a context, and the timed loops over it."""
+
+    def __init__(self, torch, shape, weights, lens, room, dev, rank, dist, dist_dev, opts=()):
+        from paper_2410_12513_b200 import FirstContext, KVCache
+        self.torch, self.shape, self.lens, self.dev, self.dist, self.dist_dev = torch, shape, lens, dev, dist, dist_dev
+        s, L, B = shape, shape.n_layers, len(lens)
+        self.B, self.L = B, L
+        g = torch.Generator(device=dev)
+        g.manual_seed(4321 + rank)
+        caps = (lens + room + 1).astype(np.int32)
+        off = np.concatenate([[0], np.cumsum(caps[:-1], dtype=np.int64)]).astype(np.int64)
+        tot = int(caps.sum())
+        self.caps = caps
+
+        def rnd(shp):
+            t = torch.empty(shp, dtype=torch.bfloat16, device=dev)
+            t.normal_(0.0, 1.0, generator=g)
+            return t
+
+        self.kk = [rnd((s.n_kv_heads, tot, s.head_dim)) for _ in range(L)]
+        self.vv = [rnd((s.n_kv_heads, tot, s.head_dim)) for _ in range(L)]
+        self.len0 = torch.from_numpy(np.broadcast_to(lens.astype(np.int32), (L, B)).copy()).to(dev)
+        self.pos0 = torch.from_numpy(lens.astype(np.int32)).to(dev)
+        self.len_t, self.pos_t = self.len0.clone(), self.pos0.clone()
+        self.kv = KVCache(self.kk, self.vv, torch.from_numpy(off).to(dev), torch.from_numpy(caps).to(dev),
+                          self.len_t, self.pos_t)
+        self.ctx = FirstContext(shape, 1, B, int(caps.max()), weights)
+        for o in opts:
+            name, val = o.split("=")
+            self.ctx.set_option(name, int(val))
+        self.tok0 = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).to(dev)
+        self.tok_a, self.tok_b = self.tok0.clone(), self.tok0.clone()
+        self.stream = torch.cuda.current_stream()
+
+    def close(self):
+        self.ctx.close()
+        self.kk = self.vv = self.kv = None
+        self.torch.cuda.empty_cache()
+
+    def reset(self):
+        self.len_t.copy_(self.len0)
+        self.pos_t.copy_(self.pos0)
+        self.tok_a.copy_(self.tok0)
+
+    def steps(self, n):
+        a, b = self.tok_a, self.tok_b
+        for _ in range(n):
+            self.ctx.decode_step(a, self.kv, None, b)
+            a, b = b, a
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
+
+    def timed(self, mask, K, W):
+        """W untimed + exactly K timed steps under `mask` (numpy [B][L]); -> (ms of the K steps, max over
+        ranks; launches)."""
+        torch = self.torch
+        self.ctx.set_mask(torch.from_numpy(np.ascontiguousarray(mask)).to(self.dev))
+        self.reset()
+        self.steps(W)
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = self.ctx.launch_count()
+        e0.record(self.stream)
+        self.steps(K)
+        e1.record(self.stream)
+        self.barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1), self.dist, self.dist_dev)
+        return ms, self.ctx.launch_count() - l0
+
+    def in_step_ms(self, mask, n=8):
+        """Where a step's time goes while it runs the way it is timed (one graph, dependent launches overlapping):
+        every launch stamps first-CTA start / last-warp end; per class, the time from the previous launch's end to
+        this launch's end, summed -- the classes add up to the step.  Mean over n steps, ms."""
+        torch = self.torch
+        self.ctx.set_mask(torch.from_numpy(np.ascontiguousarray(mask)).to(self.dev))
+        self.ctx.set_option("stamp", 1)
+        self.reset()
+        self.steps(3)
+        excl, span, cnt = {}, {}, {}
+        total = 0.0
+        for _ in range(n):
+            self.steps(1)
+            tr = self.ctx.step_trace()
+            prev_end = tr[0][1]
+            for name, t0, t1 in tr:
+                excl[name] = excl.get(name, 0.0) + max(0, t1 - prev_end) / 1e6
+                span[name] = span.get(name, 0.0) + (t1 - t0) / 1e6
+                cnt[name] = cnt.get(name, 0) + 1
+                prev_end = max(prev_end, t1)
+            total += (prev_end - tr[0][1]) / 1e6
+        self.ctx.set_option("stamp", 0)
+        return ({k: v / n for k, v in excl.items()}, {k: v / n for k, v in span.items()},
+                {k: v // n for k, v in cnt.items()}, total / n)
+
+
+def fractions(bm, ms_step, peak):
+    return {"bytes_strict": bm["strict"], "bytes_full": bm["full"],
+            "frac_strict_of_measured": bm["strict"] / (ms_step * 1e6) / peak,
+            "frac_full_of_measured": bm["full"] / (ms_step * 1e6) / peak,
+            "frac_strict_of_8TBps": bm["strict"] / (ms_step * 1e6) / 8000.0,
+            "floor_ms_strict_measured_peak": bm["strict"] / peak / 1e6}
+
+
+def sub_record(torch, name, weights_for, dev, rank, dist, dist_dev, peak, opts, K, W, sweep=False):
+    """A compact record of another workload of the benchmark set, measured the same way (W + exactly K steps,
+    CUDA events): routed and all-keep step time, bytes and roofline fractions; for the sweep config the six
+    skip fractions with aligned and independent masks."""
+    wl = WORKLOADS[name]
+    shape = SHAPES[wl["shape"]]
+    B, L = wl["B"], shape.n_layers
+    lens = fi.prompt_lengths(B, wl["lo"], wl["hi"], 1000 + rank)
+    mask = make_mask(wl["mask"], B, L, 2000 + rank)
+    job = Job(torch, shape, weights_for(wl["shape"]), lens, W + K, dev, rank, dist, dist_dev, opts)
+    mid = lens + W + K // 2
+    try:
+        ms, launches = job.timed(mask, K, W)
+        dense_ms, _ = job.timed(np.ones_like(mask), K, W)
+        bm, bmd = byte_model(shape, mask, mid), byte_model(shape, np.ones_like(mask), mid)
+        rec = {"workload": name, "shape": wl["shape"], "batch": B, "prompt_lengths": [int(lens.min()), int(lens.max())],
+               "mask": list(wl["mask"]), "skip_fraction": float(1 - mask.mean()), "steps": K, "warmup": W,
+               "ms_per_step": ms / K, "tokens_per_s": job_tokens_per_s(1 if dist is None else dist.get_world_size(), B, K, ms),
+               "gpu_launches_per_step": launches / K, **fractions(bm, ms / K, peak),
+               "dense": {"ms_per_step": dense_ms / K, "bytes_strict": bmd["strict"],
+                         "latency_ratio_routed_over_dense": ms / dense_ms,
+                         "bytes_ratio_routed_over_dense": bm["full"] / bmd["full"]}}
+        if sweep:
+            rows = []
+            for frac in (0.0, 0.1, 0.2, 0.3, 0.4, 0.5):
+                row = {"skip": frac}
+                for kind in ("aligned", "independent"):
+                    mk = fi.mask_aligned(B, L, frac) if kind == "aligned" else fi.mask_independent(B, L, frac, 3000 + rank)
+                    t, _ = job.timed(mk, K, W)
+                    b_ = byte_model(shape, mk, mid)
+                    row[kind] = {"ms_per_step": t / K, "bytes_strict": b_["strict"],
+                                 "frac_strict_of_measured": b_["strict"] / (t / K * 1e6) / peak,
+                                 "latency_over_all_keep": (t / K) / (dense_ms / K)}
+                rows.append(row)
+            rec["skip_sweep"] = rows
+        if job.ctx.device_flags():
+            raise RuntimeError(f"device flags set during sub-record {name}")
+        return rec
+    finally:
+        job.close()
+
+
+def run_cuda(args, wl, shape, mask, lens):
+    import torch
+    from paper_2410_12513_b200 import FirstContext
+
+    rank, world, local, dist, dist_dev = init_replica()
+    dev = torch.device("cuda", local)
+    B, L, K, W = mask.shape[0], shape.n_layers, args.steps, args.warmup
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234 + rank)
+    s = shape
+    w_cache = {}
+
+    def weights_for(shape_key):
+        if shape_key not in w_cache:
+            w_cache.clear()  # one model resident at a time
+            torch.cuda.empty_cache()
+            w_cache[shape_key] = make_weights_dev(torch, shape if shape_key == wl["shape"] else SHAPES[shape_key], dev, g)
+        return w_cache[shape_key]
+
+    weights = weights_for(wl["shape"])
+    job = Job(torch, shape, weights, lens, W + K, dev, rank, dist, dist_dev, args.opt)
+    ctx, kv, caps, stream = job.ctx, job.kv, job.caps, job.stream
+    peaks = {}
+    try:
+        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
+    except Exception:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
 
     if args.prefill_only:
         if rank == 0:
-            peaks = {}
-            try:
-                peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
-            except Exception:
-                pass
             print(json.dumps({"prefill_only": True, "layers": L, "options": args.opt,
                               "prefill": prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, opts=args.opt),
                               "note": "profiling case, not a benchmark value"}))
         return
 
-    tok0 = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).to(dev)
-    tok_a, tok_b = tok0.clone(), tok0.clone()
-    mask_t = torch.from_numpy(mask).to(dev)
-    dense_t = torch.ones_like(mask_t)
-
-    def reset():
-        len_t.copy_(len0)
-        pos_t.copy_(pos0)
-        tok_a.copy_(tok0)
-
-    def steps(n):
-        a, b = tok_a, tok_b
-        for _ in range(n):
-            ctx.decode_step(a, kv, None, b)
-            a, b = b, a
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    def timed(mask_dev):
-        ctx.set_mask(mask_dev)
-        reset()
-        steps(W)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        l0 = ctx.launch_count()
-        e0.record(stream)
-        steps(K)
-        e1.record(stream)
-        barrier()
-        ms = e0.elapsed_time(e1)
-        launches = ctx.launch_count() - l0
-        ms = max_over_ranks(ms, dist, dev)
-        return ms, launches
-
     # ---- routing + plan, once per batch (reported, not part of the step)
     route = None
-    if rank == 0 and not args.no_route:
+    if rank == 0 and not args.no_route and not args.quick:
         n_tok = int(lens.sum())
-        hid = rnd((n_tok, s.d_model), 1.0)
+        hid = torch.empty((n_tok, s.d_model), dtype=torch.bfloat16, device=dev)
+        hid.normal_(0.0, 1.0, generator=g)
         cu = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).to(dev)
         rw = 0.02 * torch.randn(s.d_model, device=dev, generator=g)
         rmask = torch.zeros((B, L), dtype=torch.uint8, device=dev)
         for _ in range(3):
-            ctx.prefill_route(0, hid, cu, rw, None, 0.5, 1, rmask)
+            ctx.prefill_route(0, hid, cu, rw, None, 0.5, 0, rmask)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         reps = 10
         for i in range(reps):
-            ctx.prefill_route(i % L, hid, cu, rw, None, 0.5, 1, rmask)
+            ctx.prefill_route(i % L, hid, cu, rw, None, 0.5, 0, rmask)
         e1.record(stream)
         torch.cuda.synchronize()
         rms = e0.elapsed_time(e1) / reps
-        route = {"ms_per_layer": rms, "hidden_bytes": n_tok * s.d_model * 2,
+        route = {"ms_per_layer": rms, "hidden_bytes": n_tok * s.d_model * 2, "router_mode": "mean of per-token sigmoids",
                  "GBps": n_tok * s.d_model * 2 / rms / 1e6, "tokens": n_tok}
         del hid
 
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(physical_gpu_index(local))
     with sampler:
-        ms_total, launches = timed(mask_t)
+        ms_total, launches = job.timed(mask, K, W)
     clocks = sampler.summary()
     ms_step = ms_total / K
     value = job_tokens_per_s(world, B, K, ms_total)
@@ -396,27 +567,27 @@ def run_cuda(args, wl, shape, mask, lens):
             print(json.dumps({"quick": True, "ms_per_step": ms_step, "value": value, "layers": L,
                               "gpu_launches": int(launches), "note": "profiling case, not a benchmark value"}))
         return
-    dense_ms, dense_launches = timed(dense_t)
+    dense_ms, dense_launches = job.timed(np.ones_like(mask), K, W)
     dense_ms /= K
-    repeat_ms, _ = timed(mask_t)  # the routed run once more, after the dense one (order effects show here)
+    repeat_ms, _ = job.timed(mask, K, W)  # the routed run once more, after the dense one (order effects show here)
     repeat_ms /= K
 
-    # Step latency against the skip rate, on this workload's batch and caches: always a short version (three
-    # rates, both mask structures), the six rates of the sweep config with --sweep.
+    # Step latency against the skip rate, on this workload's batch and caches: a short version (three rates, both
+    # mask structures); the six rates on this workload with --sweep (the sweep config itself is a sub-record).
     sweep = []
-    if True:
-        for frac in ((0.0, 0.1, 0.2, 0.3, 0.4, 0.5) if args.sweep else (0.0, 0.25, 0.5)):
-            row = {"skip": frac}
-            for kind in ("aligned", "independent"):
-                mk = fi.mask_aligned(B, L, frac) if kind == "aligned" else fi.mask_independent(B, L, frac, 3000 + rank)
-                ms, _ = timed(torch.from_numpy(mk).to(dev))
-                bmk = byte_model(shape, mk, lens + W + K // 2)
-                row[kind] = {"ms_per_step": ms / K, "bytes_strict": bmk["strict"]}
-            sweep.append(row)
+    for frac in ((0.0, 0.1, 0.2, 0.3, 0.4, 0.5) if args.sweep else (0.0, 0.25, 0.5)):
+        row = {"skip": frac}
+        for kind in ("aligned", "independent"):
+            mk = fi.mask_aligned(B, L, frac) if kind == "aligned" else fi.mask_independent(B, L, frac, 3000 + rank)
+            ms, _ = job.timed(mk, K, W)
+            bmk = byte_model(shape, mk, lens + W + K // 2)
+            row[kind] = {"ms_per_step": ms / K, "bytes_strict": bmk["strict"]}
+        sweep.append(row)
 
     # ---- end to end through the public call with host buffers
-    ctx.set_mask(mask_t)
-    reset()
+    ctx.set_mask(torch.from_numpy(mask).to(dev))
+    job.reset()
+    tok_a, tok_b = job.tok_a, job.tok_b
     h_tok = torch.from_numpy(fi.tokens(shape, B, 7 + rank)).pin_memory()
     h_next = torch.empty(B, dtype=torch.int32).pin_memory()
 
@@ -429,50 +600,41 @@ def run_cuda(args, wl, shape, mask, lens):
             h_tok.copy_(h_next)
 
     e2e_steps(W)
-    barrier()
+    job.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     e2e_steps(K)
     e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    job.barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dist_dev)
     e2e = {"value": job_tokens_per_s(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": B * 4,
            "d2h_bytes_per_step": B * 4, "ms_per_step": e2e_ms / K}
 
-    # ---- per-kernel-class device time (separate pass: event pairs around every launch)
-    reset()
-    steps(2)
+    # ---- where the step's time goes: in-step stamps (nothing serialised), then event pairs (serialised)
+    excl_ms, span_ms, cls_launches, traced_step_ms = job.in_step_ms(mask)
+    ctx.set_mask(torch.from_numpy(mask).to(dev))
+    job.reset()
+    job.steps(2)
     torch.cuda.synchronize()
     kp = min(K, 16)
     ctx.profile(True)
-    steps(kp)
+    job.steps(kp)
     prof = ctx.profile_read()
     ctx.profile(False)
     flags = ctx.device_flags()
     if flags:
         raise RuntimeError(f"device flags set during the benchmark: {flags}")
-    if rank != 0:
-        return
 
     mid_lens = lens + W + K // 2
     bm = byte_model(shape, mask, mid_lens)
     bm_dense = byte_model(shape, np.ones_like(mask), mid_lens)
-    peaks = {}
-    try:
-        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
-    except Exception:
-        pass
-    peak = float(peaks.get("hbm_gbs", 6650.0))
-    peak_kind = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
     cls_ms = {k: v[0] / kp for k, v in prof.items() if v[1]}
-    tot_cls = sum(cls_ms.values())
     cnt = mask.sum(0)
     proj_bytes = bm["weights"] + bm["lm_head"]
     alg = {"gemv_rows": proj_bytes, "gemm_tc": proj_bytes, "attn_split": bm["kv"]}
     if cls_ms.get("gemv_rows") and cls_ms.get("gemm_tc"):
         alg = {"attn_split": bm["kv"]}  # projections split over two classes: attribute by class below
-    dom = max(cls_ms, key=cls_ms.get)
+    dom = max(excl_ms, key=excl_ms.get)
     traffic = None
     try:  # DRAM bytes of the projection launches from the committed ncu capture, if the kernel is unchanged since
         import hashlib
@@ -485,17 +647,23 @@ def run_cuda(args, wl, shape, mask, lens):
         traffic = None
     roof = {"bound": "hbm", "kernel": dom, "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "traffic": traffic,
             "traffic_note": "per step, scaled from the 2-layer ncu capture in profiles/ (per launch x launches)" if traffic else None,
-            "ms_per_step": cls_ms[dom], "share_of_kernel_time": cls_ms[dom] / tot_cls,
-            "timing": "CUDA event pair around every launch of the class, summed over a profiled pass of the timed steps; "
-                      "the events serialise the launches, so the overlap between neighbouring kernels that a normal step "
-                      "has (weight tiles requested before the dependency wait) is absent: a lower bound on the in-step rate"}
+            "ms_per_step": excl_ms[dom], "share_of_step": excl_ms[dom] / max(traced_step_ms, 1e-9),
+            "launches_per_step": cls_launches.get(dom),
+            "timing": "in-step: every launch stamps its first CTA's start and last warp's end (global ns timer) while the "
+                      "step runs as timed (one CUDA graph, dependent launches overlapping); a class's time is the sum, over "
+                      "its launches, of (this launch's end - previous launch's end), so the classes add up to the step",
+            "ms_per_step_event_pairs": cls_ms.get(dom),
+            "event_pairs_note": "CUDA event pair around every launch (serialises the step: an upper bound on the class's time)"}
     if dom in alg:
-        roof["achieved"] = alg[dom] / cls_ms[dom] / 1e6
+        roof["achieved"] = alg[dom] / excl_ms[dom] / 1e6
         roof["frac"] = roof["achieved"] / peak
         roof["algorithmic_bytes_per_step"] = alg[dom]
     else:
         roof["achieved"] = None
         roof["frac"] = None
+    in_step = {k: {"ms": excl_ms[k], "span_ms": span_ms[k], "launches": cls_launches[k],
+                   **({"GBps": alg[k] / excl_ms[k] / 1e6, "frac_of_measured": alg[k] / excl_ms[k] / 1e6 / peak}
+                      if k in alg and excl_ms[k] > 0 else {})} for k in excl_ms}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -508,23 +676,32 @@ def run_cuda(args, wl, shape, mask, lens):
                       **({"layers": L, "note": "reduced layer count: not a benchmark value"} if args.layers else {})},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
            "roofline": roof,
-           "step_roofline": {"bytes_strict": bm["strict"], "bytes_full": bm["full"],
-                             "frac_strict_of_measured": bm["strict"] / (ms_step * 1e6) / peak,
-                             "frac_full_of_measured": bm["full"] / (ms_step * 1e6) / peak,
-                             "frac_strict_of_8TBps": bm["strict"] / (ms_step * 1e6) / 8000.0,
-                             "floor_ms_strict_measured_peak": bm["strict"] / peak / 1e6},
+           "step_roofline": fractions(bm, ms_step, peak),
            "dense": {"ms_per_step": dense_ms, "gpu_launches": int(dense_launches), "bytes_strict": bm_dense["strict"],
                      "latency_ratio_routed_over_dense": ms_step / dense_ms,
                      "bytes_ratio_routed_over_dense": bm["full"] / bm_dense["full"]},
            "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
-           "kernel_ms_per_step": cls_ms, "route": route}
-    if not args.no_prefill:
+           "kernel_ms_in_step": in_step, "traced_step_ms": traced_step_ms,
+           "kernel_ms_per_step_event_pairs": cls_ms, "route": route}
+    if not args.no_prefill and rank == 0:
         out["prefill"] = prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, opts=args.opt)
-    if not args.no_cpu_baseline:
-        out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5, rows=min(B, 32), layers=4)
-        out["cpu_baseline"].pop("ms_per_step", None)
-    print(json.dumps(out))
+    job.close()
+    if not args.no_sub and not args.layers and not args.opt and args.workload == "cfg2_8b_b32":
+        # the other workloads of the benchmark set, each measured the same way (every rank runs them: replicas)
+        subs = {}
+        for name, k_sub, sweep_sub in (("cfg4_8b_b64", 32, True), ("cfg3_8b_b256", 32, False), ("cfg1_1b_b1", 128, False)):
+            try:
+                subs[name] = sub_record(torch, name, weights_for, dev, rank, dist, dist_dev, peak, args.opt, k_sub, 5, sweep_sub)
+            except Exception as e:  # a sub-record never takes the main line down
+                subs[name] = {"error": f"{type(e).__name__}: {e}"[:300]}
+        out["workloads"] = subs
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            out["cpu_baseline"] = oracle_sample(shape, mask, lens, 5, rows=min(B, 32), layers=4)
+            out["cpu_baseline"].pop("ms_per_step", None)
+        print(json.dumps(out))
     if dist is not None:
+        dist.barrier()
         dist.destroy_process_group()
 
 
@@ -546,6 +723,7 @@ def main():
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
     ap.add_argument("--sweep", action="store_true",
                     help="time six skip fractions 0..50 %% (aligned and independent masks) on this workload instead of three")
+    ap.add_argument("--no-sub", action="store_true", help="skip the sub-records of the other benchmark workloads")
     ap.add_argument("--quick", action="store_true",
                     help="only the main timed loop (for profiler captures): no dense/e2e/per-kernel legs")
     args = ap.parse_args()
@@ -555,6 +733,9 @@ def main():
         wl["mask"] = tuple([parts[0]] + [float(x) for x in parts[1:]])
     if args.steps is None:
         args.steps = 64 if args.impl == "cuda" else 2
+    if args.impl == "cuda" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under torchrun: start the N replicas here, one process per GPU
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))
     if args.impl == "cuda" and not args.quick:
         args.warmup = max(args.warmup, 3)
     shape = SHAPES[wl["shape"]]

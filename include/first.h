@@ -291,6 +291,15 @@ int first_sample_topk(const float *logits, int32_t B, int32_t vocab, int32_t top
  * *flags = 0, or FIRST_E_DEVICE_FLAG with the FIRST_FLAG_* bits in *flags. */
 int first_last_device_flags(first_ctx *ctx, uint32_t *flags, void *stream);
 
+/* Self-test of the bounded waits (the paper has no counterpart).  Every wait on a copy or on another role
+ * inside the kernels gives up after a fixed number of polls, raises FIRST_FLAG_WAIT_EXPIRED and lets the
+ * kernel end; a step in which that happened has undefined outputs (first_last_device_flags then also
+ * clears the attention merge counters, so later steps are sound).  This call runs that give-up path on
+ * purpose, harmlessly: one thread waits `polls` (1 .. 2^20) times on a barrier nothing will ever complete,
+ * with no copy in flight.  *returned = what the wait reported (0 = gave up), *abort_word = the CTA's abort
+ * word (1); the context's flag word gets FIRST_FLAG_WAIT_EXPIRED.  Waits for `stream`. */
+int first_selftest_wait_expiry(first_ctx *ctx, int32_t polls, int32_t *returned, int32_t *abort_word, void *stream);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t first_launch_count(const first_ctx *ctx);
 
@@ -305,6 +314,18 @@ int first_profile(first_ctx *ctx, int32_t enable);
 int first_profile_read(first_ctx *ctx, int32_t n, double *ms, int64_t *launches, void *stream);
 int32_t first_kernel_class_count(void);
 const char *first_kernel_class_name(int32_t k);
+
+/* Measurement aid (the paper has no counterpart): where a step's time goes WITHOUT serialising it.
+ * With option "stamp" = 1 every kernel of a step records, in device memory, when its first CTA
+ * started and when its last warp ended (global nanosecond timer); the step runs as it always does
+ * (one CUDA graph, programmatic dependent launch).  first_step_trace waits for `stream` and copies
+ * out the last step's launches in launch order: cls[i] = kernel class (first_kernel_class_name),
+ * t_start[i], t_end[i] in nanoseconds of one clock.  The time from launch i-1's end to launch i's
+ * end, summed per class, splits the step's duration among the classes without double counting.
+ * Steps with more than 2048 launches are truncated.  Host arrays of max_n entries; *n_out = entries
+ * written.  Errors: FIRST_E_ARG, FIRST_E_STATE (option off), FIRST_E_CUDA. */
+int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_start, uint64_t *t_end,
+                     int32_t *n_out, void *stream);
 
 /* Options (A/B measurements and tuning).  A negative value restores the default.
  *   "max_gemv_rows"  largest active-row count served by the CUDA-core GEMV path; layers with
@@ -336,6 +357,7 @@ const char *first_kernel_class_name(int32_t k);
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
  *                    its epilogue (needs ffn_dim % 64 == 0).
+ *   "stamp"          1 = record per-launch start/end times for first_step_trace (default 0)
  *   "use_pdl"        0 = kernels of a step are launched strictly one after another.  Default 1:
  *                    programmatic dependent launch lets a kernel's prologue (and, for the
  *                    projections, its first weight tiles) overlap the previous kernel's tail.

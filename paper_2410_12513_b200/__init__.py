@@ -8,9 +8,9 @@ the compiled library or without a CUDA device the calls raise.
 """
 from .binding import (FirstContext, FirstError, KVCache, first_create, first_decode_step, first_destroy,
                       first_get_plan, first_last_device_flags, first_prefill, first_prefill_route, first_prefill_route_static, first_profile, first_profile_read, first_sample_topk, first_set_mask,
-                      first_set_option, first_set_sampling, lib, library_path)
+                      first_set_option, first_set_sampling, first_step_trace, lib, library_path)
 
 __all__ = ["FirstContext", "FirstError", "KVCache", "first_create", "first_decode_step", "first_destroy",
            "first_get_plan", "first_last_device_flags", "first_prefill", "first_prefill_route", "first_prefill_route_static", "first_profile",
            "first_profile_read", "first_sample_topk", "first_set_mask",
-           "first_set_option", "first_set_sampling", "lib", "library_path"]
+           "first_set_option", "first_set_sampling", "first_step_trace", "lib", "library_path"]

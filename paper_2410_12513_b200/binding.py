@@ -86,6 +86,10 @@ def lib():
         L.first_profile.restype = C.c_int
         L.first_profile_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_profile_read.restype = C.c_int
+        L.first_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.first_selftest_wait_expiry.restype = C.c_int
+        L.first_step_trace.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.first_step_trace.restype = C.c_int
         L.first_kernel_class_count.restype = C.c_int32
         L.first_kernel_class_name.restype = C.c_char_p
         L.first_kernel_class_name.argtypes = [C.c_int32]
@@ -293,6 +297,20 @@ def first_profile_read(h, stream=None):
     return {lib().first_kernel_class_name(k).decode(): (ms[k], cnt[k]) for k in range(n)}
 
 
+def first_step_trace(h, stream=None, max_n=2048):
+    """Launches of the last step with option "stamp" on: [(class name, start_ns, end_ns)] in launch order."""
+    import numpy as np
+    cls = np.zeros(max_n, dtype=np.int32)
+    t0 = np.zeros(max_n, dtype=np.uint64)
+    t1 = np.zeros(max_n, dtype=np.uint64)
+    n = C.c_int32(0)
+    rc = lib().first_step_trace(h, max_n, cls.ctypes.data, t0.ctypes.data, t1.ctypes.data, C.byref(n), _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_step_trace")
+    names = [lib().first_kernel_class_name(int(k)).decode() for k in cls[:n.value]]
+    return [(names[i], int(t0[i]), int(t1[i])) for i in range(n.value)]
+
+
 class FirstContext:
     """Owns one library context; methods mirror the C calls."""
 
@@ -343,6 +361,17 @@ class FirstContext:
     def set_sampling(self, top_k, temperature, uniforms):
         self._uniforms = uniforms  # borrowed by the library until the next call
         first_set_sampling(self.h, top_k, temperature, uniforms)
+
+    def selftest_wait_expiry(self, polls=1000, stream=None):
+        """Runs a bounded wait that must give up; -> (what the wait returned, the abort word)."""
+        r, a = C.c_int32(-1), C.c_int32(-1)
+        rc = lib().first_selftest_wait_expiry(self.h, int(polls), C.byref(r), C.byref(a), _stream(stream))
+        if rc:
+            raise FirstError(rc, "first_selftest_wait_expiry")
+        return r.value, a.value
+
+    def step_trace(self, stream=None):
+        return first_step_trace(self.h, stream)
 
     def profile(self, enable):
         first_profile(self.h, enable)

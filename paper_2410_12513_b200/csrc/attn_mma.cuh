@@ -83,7 +83,10 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                                                       uint32_t* __restrict__ ticket, float* __restrict__ out,
                                                       __nv_bfloat16* __restrict__ out_hi,
                                                       __nv_bfloat16* __restrict__ out_lo,
-                                                      uint32_t* __restrict__ flags, const RopeFuse rf) {
+                                                      uint32_t* __restrict__ flags, const RopeFuse rf,
+                                                      const __grid_constant__ tc::NextWeights nx,
+                                                      uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     constexpr int kHalves = HD / 64;              // 128-byte column groups per row
     constexpr int kBox = kTile * 128;             // bytes of one 64-token x 64-element box
     constexpr int kStageBytes = 2 * kHalves * kBox;
@@ -110,6 +113,12 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     }
     __syncthreads();
     pdl_wait();
+    if (threadIdx.x == 129) {
+        // This kernel is latency-bound and leaves about half of the HBM bandwidth unused: one thread per CTA
+        // (work items that turn out empty included) asks for the first weight tiles of the next projection.
+        const int cta = (int)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x);
+        tc::prefetch_next_weights(nx, cta, (int)(gridDim.x * gridDim.y * gridDim.z));
+    }
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
     const longlong2 ri = __ldcg(&rowinfo[i]);
@@ -150,11 +159,13 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
                     tc::tma_load_2d_hint(sa + (kHalves + hf) * kBox, &tmV, full_bar(s), hf * 64, row, pol);
                 }
             }
-            if (abort_s) {
-                for (int j = max(0, issued - kStages); j < issued; ++j) {
-                    const uint32_t bar = full_bar(j % kStages), ph = (uint32_t)(j / kStages) & 1u;
-                    for (uint32_t it = 0; it < tc::kSpinLimit && !tc::mbar_try_wait(bar, ph); ++it) {}
-                }
+            // The producer leaves only when every copy it issued has landed (the last use of each stage), whether
+            // or not a role has given up and whoever noticed first.  A CTA's shared memory is released when all
+            // of its threads have left, this one included, so it is never reused with a copy in flight.  The
+            // consumers wait for the same barriers in a normal run, so this costs nothing.
+            for (int j = max(0, issued - kStages); j < issued; ++j) {
+                const uint32_t bar = full_bar(j % kStages), ph = (uint32_t)(j / kStages) & 1u;
+                for (uint32_t it = 0; it < tc::kSpinLimit && !tc::mbar_try_wait(bar, ph); ++it) {}
             }
         }
         return;

@@ -17,7 +17,9 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
                                                          const int32_t* len_l,
                                                          const int32_t* __restrict__ slab_cap,
                                                          const int32_t* __restrict__ idx, int Hq,
-                                                         float* __restrict__ o_part, float2* __restrict__ ml_part) {
+                                                         float* __restrict__ o_part, float2* __restrict__ ml_part,
+                                                         uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     constexpr int EPL = HD / 32;
@@ -96,7 +98,9 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
 // optionally, its bfloat16 hi/lo split for the tensor-core O-projection.
 __global__ void __launch_bounds__(128) attn_combine(const float* o_part, const float2* ml_part,
                                                     int S, int HD, float* __restrict__ out,
-                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                    uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const size_t hq = blockIdx.x;  // flat (row, query head)

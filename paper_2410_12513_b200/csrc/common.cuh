@@ -26,6 +26,26 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 // kernel parameter): pointers to data produced inside a step therefore carry no __restrict__.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// In-step timing aid (off unless asked for): every CTA folds its entry time into the launch's
+// first-start word and every warp its exit time into the launch's last-end word, both read from
+// the global nanosecond timer.  `slot` points at the start word; the end word sits kStampCap
+// words further on.  A null slot costs one predictable branch.
+constexpr int kStampCap = 2048;
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+struct Stamp {
+    unsigned long long* slot;
+    __device__ __forceinline__ explicit Stamp(uint64_t* s) : slot(reinterpret_cast<unsigned long long*>(s)) {
+        if (slot && threadIdx.x == 0 && threadIdx.y == 0) atomicMin(slot, global_ns());
+    }
+    __device__ __forceinline__ ~Stamp() {
+        if (slot && (threadIdx.x & 31) == 0) atomicMax(slot + kStampCap, global_ns());
+    }
+};
+
 // two packed bfloat16 -> two float32 (a bfloat16 is the upper half of a float32)
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }

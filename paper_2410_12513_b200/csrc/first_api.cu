@@ -89,7 +89,15 @@ struct first_ctx {
     int use_graph = 1;
     int use_pdl = 1;
     bool pdl_next = false;  // the next kernel launch may overlap its predecessor (programmatic dependent launch)
+    // in-step timing (option "stamp"): first-CTA start / last-warp end of every launch of a step
+    int stamp_on = 0;
+    uint64_t* stamps = nullptr;  // [2][kStampCap]: starts, ends
+    int stamp_n = 0;
+    std::vector<int> stamp_cls;
     // options
+    int pf_depth = 0;       // k-blocks per work unit of the next projection that a projection's idle producer prefetches
+    int pf_attn_depth = 0;  // the same for the attention kernel (head of the gate/up weights)
+    int pf_o = 0;           // the QKV projection prefetches the whole O matrix
     int max_gemv_rows = -1;
     int attn_simple = -1;
     int tc_use_lo = 1;
@@ -157,6 +165,13 @@ struct Launch {
     }
 };
 
+// Timing slot of the next launch of a step (NULL while in-step timing is off or the table is full).
+uint64_t* stamp_slot(first_ctx* c, int cls) {
+    if (!c->stamp_on || !c->stamps || c->stamp_n >= kStampCap) return nullptr;
+    c->stamp_cls.push_back(cls);
+    return c->stamps + c->stamp_n++;
+}
+
 #define FIRST_LAUNCH(cls, ...)      \
     do {                            \
         Launch guard_(c, st, cls);  \
@@ -181,7 +196,13 @@ int launch_k(first_ctx* c, cudaStream_t st, int cls, void (*kern)(P...), dim3 gr
     cfg.attrs = at;
     cfg.numAttrs = (c->use_pdl && !c->profiling && c->pdl_next) ? 1 : 0;
     c->pdl_next = true;
-    CU_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...));
+    if constexpr (sizeof...(A) + 1 == sizeof...(P)) {
+        // the kernel's last parameter is its in-step timing slot
+        uint64_t* stamp = stamp_slot(c, cls);
+        CU_TRY(cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)..., stamp));
+    } else {
+        CU_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...));
+    }
     return FIRST_OK;
 }
 
@@ -252,48 +273,95 @@ int tc_ksplit(const first_ctx* c, int tiles, int K, int epi, int m, int slots) {
     return 1;
 }
 
+// Launch shape of one tensor-core projection of mm (<= 256) compact rows: a pure function of the sizes and the
+// options, so that the kernel BEFORE a projection can know which weight tiles that projection will ask for first.
+struct TcShape {
+    int n_pad, use_lo, mt, tile_rows, tiles, stage_bytes, stages, ksplit, acc_cols, tmem_cols, kblocks;
+};
+TcShape tc_shape(const first_ctx* c, int n_out, int K, int mm, int epi) {
+    TcShape t{};
+    t.n_pad = (mm + 15) / 16 * 16;
+    t.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+    t.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
+    // Two weight tiles per CTA share every activation tile.  Worth it exactly when the activation tiles are
+    // so wide that only one single-tile CTA would fit per SM anyway (from 96 rows): the tile pair halves the
+    // activation bytes an SM pulls from L2 per weight byte (config 3: -4 %; 115 rows: -16 % per step);
+    // below that, two single-tile CTAs per SM overlap each other's set-up and epilogue and win.
+    const int stage1 = tc::kABytes + t.n_pad * 128 * (t.use_lo ? 2 : 1);
+    if (c->tc_mt2_min_rows >= 0) t.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
+    else t.mt = (3 * stage1 > c->tc_smem_kb * 1024) ? 2 : 1;
+    if (epi == tc::kEpiSwiglu && n_out % 128) t.mt = 1;
+    t.tile_rows = epi == tc::kEpiSwiglu ? (t.mt == 1 ? c->pair_rows : 128) : tc::kBlockM * t.mt;
+    t.tiles = (n_out + t.tile_rows - 1) / t.tile_rows;
+    t.stage_bytes = tc::kABytes * t.mt + t.n_pad * 128 * (t.use_lo ? 2 : 1);
+    const int budget = (3 * t.stage_bytes <= c->tc_smem_kb * 1024) ? c->tc_smem_kb * 1024 : 200 * 1024;
+    const bool one_per_sm = budget != c->tc_smem_kb * 1024;
+    t.stages = std::max(1, std::min(8, budget / t.stage_bytes));
+    t.ksplit = tc_ksplit(c, t.tiles, K, epi, mm, c->n_sm * (one_per_sm ? 1 : 2));
+    int cols = 32;
+    while (cols < t.n_pad) cols *= 2;
+    t.acc_cols = cols;
+    t.tmem_cols = std::max(32, cols * t.mt);
+    return t;
+}
+
+// What the projection (weights tm / tm_pair, n_out x K, m rows, epilogue epi) will read first: handed to the
+// kernel that runs before it (see tc::NextWeights).  depth = k-blocks per work unit; 0 rows or depth: nothing.
+tc::NextWeights next_weights(const first_ctx* c, const CUtensorMap* tm, const CUtensorMap* tm_pair, int n_out, int K,
+                             int m, int epi, int depth) {
+    tc::NextWeights nx{};
+    if (!tm || m <= 0 || m > 256 || depth <= 0) return nx;
+    const TcShape t = tc_shape(c, n_out, K, m, epi);
+    const bool pairs = epi == tc::kEpiSwiglu;
+    nx.map = (pairs && t.mt == 1) ? *tm_pair : *tm;
+    nx.mode = pairs ? 2 : 1;
+    nx.tiles = t.tiles;
+    nx.ksplit = t.ksplit;
+    nx.kblocks = t.kblocks;
+    nx.depth = depth;
+    nx.rows = pairs ? t.tile_rows : tc::kBlockM;
+    nx.n_out = n_out;
+    nx.mt = t.mt;
+    if (pairs && t.mt == 2) {  // two 128-row boxes per half: gate rows tile*128.., up rows n_out + tile*128..
+        nx.rows = 128;
+    }
+    return nx;
+}
+
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
 //   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
 //   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
+// nx: the weights the next projection of the step reads first (prefetched into L2 by this one's idle producer).
 int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmA2, int n_out, int K,
                    const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
                    const int32_t* idx, bool pre_zeroed, float* act = nullptr, __nv_bfloat16* act_hi = nullptr,
-                   __nv_bfloat16* act_lo = nullptr) {
+                   __nv_bfloat16* act_lo = nullptr, const tc::NextWeights* nx = nullptr) {
     int rc;
+    static const tc::NextWeights kNone{};
     for (int r0 = 0; r0 < m; r0 += 256) {
         const int mm = std::min(256, m - r0);
+        const TcShape t = tc_shape(c, n_out, K, mm, epi);
         tc::GemmParams p{};
         p.n_out = n_out; p.K = K; p.m = mm;
-        p.n_pad = (mm + 15) / 16 * 16;
-        p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
-        p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
-        // Two weight tiles per CTA share every activation tile.  Worth it exactly when the activation tiles are
-        // so wide that only one single-tile CTA would fit per SM anyway (from 96 rows): the tile pair halves the
-        // activation bytes an SM pulls from L2 per weight byte (config 3: -4 %; 115 rows: -16 % per step);
-        // below that, two single-tile CTAs per SM overlap each other's set-up and epilogue and win.
-        const int stage1 = tc::kABytes + p.n_pad * 128 * (p.use_lo ? 2 : 1);
-        if (c->tc_mt2_min_rows >= 0) p.mt = (mm >= c->tc_mt2_min_rows) ? 2 : 1;
-        else p.mt = (3 * stage1 > c->tc_smem_kb * 1024) ? 2 : 1;
-        if (epi == tc::kEpiSwiglu && n_out % 128) p.mt = 1;
+        p.n_pad = t.n_pad;
+        p.kblocks = t.kblocks;
+        p.use_lo = t.use_lo;
+        p.mt = t.mt;
         p.pair_rows = c->pair_rows;
-        const int tile_rows = epi == tc::kEpiSwiglu ? (p.mt == 1 ? c->pair_rows : 128) : tc::kBlockM * p.mt;
-        const int tiles = (n_out + tile_rows - 1) / tile_rows;
+        const int tiles = t.tiles;
         p.act = act ? act + (size_t)r0 * n_out : nullptr;
         p.act_hi = act_hi ? act_hi + (size_t)r0 * n_out : nullptr;
         p.act_lo = act_lo ? act_lo + (size_t)r0 * n_out : nullptr;
-        const int stage_bytes = tc::kABytes * p.mt + p.n_pad * 128 * (p.use_lo ? 2 : 1);
-        const int budget = (3 * stage_bytes <= c->tc_smem_kb * 1024) ? c->tc_smem_kb * 1024 : 200 * 1024;
-        const bool one_per_sm = budget != c->tc_smem_kb * 1024;
-        p.stages = std::max(1, std::min(8, budget / stage_bytes));
-        p.ksplit = tc_ksplit(c, tiles, K, epi, mm, c->n_sm * (one_per_sm ? 1 : 2));
-        int cols = 32;
-        while (cols < p.n_pad) cols *= 2;
-        p.acc_cols = cols;
-        p.tmem_cols = std::max(32, cols * p.mt);
+        const int stage_bytes = t.stage_bytes;
+        p.stages = t.stages;
+        p.ksplit = t.ksplit;
+        p.acc_cols = t.acc_cols;
+        p.tmem_cols = t.tmem_cols;
         p.Y = Y ? Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy) : nullptr;
         p.ldy = ldy;
         p.idx = idx ? idx + r0 : nullptr;
         p.flags = c->flags;
+        p.stamp = stamp_slot(c, kClsGemmTc);
         CUtensorMap tmBh, tmBl;
         if ((rc = make_map(&tmBh, Xh + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
         if ((rc = make_map(&tmBl, Xl + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
@@ -311,7 +379,8 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
                     : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
                     : e == tc::kEpiSwiglu ? tc::gemm_tc_kernel<tc::kEpiSwiglu>
                                           : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
-        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(320), smem, tmA, tmA2, tmBh, tmBl, p))) return rc;
+        const tc::NextWeights& nxr = (nx && r0 + 256 >= m) ? *nx : kNone;  // the last launch of this projection
+        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(320), smem, tmA, tmA2, tmBh, tmBl, nxr, p))) return rc;
     }
     return FIRST_OK;
 }
@@ -421,7 +490,8 @@ int kv_map_for(first_ctx* c, const void* ptr, int64_t cap_total, const CUtensorM
 template <int HD, int G, bool PAIR = false>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
                        const LayerKv* kv, const void* kc, const void* vc, int C, float* out,
-                       __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale) {
+                       __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale,
+                       const tc::NextWeights& nx) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     attn::RopeFuse rf{};
     if (fuse_rope) {
@@ -433,7 +503,7 @@ int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorM
     }
     return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G, PAIR>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
                     c->rowinfo, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
-                    out_hi, out_lo, c->flags, rf);
+                    out_hi, out_lo, c->flags, rf, nx);
 }
 
 template <int HD, int G>
@@ -458,7 +528,10 @@ int attn_mma_setup(first_ctx* c) {
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const LayerKv* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
-                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair = false) {
+                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair = false,
+                    const tc::NextWeights* nxp = nullptr) {
+    static const tc::NextWeights kNone{};
+    const tc::NextWeights& nx = nxp ? *nxp : kNone;
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -480,13 +553,13 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     dim3 grid(S, d.n_kv_heads, m);
 #define FIRST_ATTN_PAIR(HD, G)                            \
     if (pair && d.head_dim == HD && c->group == G)        \
-        return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale);
+        return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale, nx);
     FIRST_ATTN_PAIR(128, 1) FIRST_ATTN_PAIR(128, 2) FIRST_ATTN_PAIR(128, 3) FIRST_ATTN_PAIR(128, 4)
     FIRST_ATTN_PAIR(64, 1) FIRST_ATTN_PAIR(64, 2) FIRST_ATTN_PAIR(64, 3) FIRST_ATTN_PAIR(64, 4)
 #undef FIRST_ATTN_PAIR
 #define FIRST_ATTN_MMA(HD, G)                 \
     if (d.head_dim == HD && c->group == G)    \
-        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale);
+        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale, nx);
     FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 3) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
     FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 3) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
@@ -500,10 +573,12 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
 template <typename WT>
 int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUtensorMap* tm, int n_out, int K,
             const float* X, const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int out_mode, float* Y,
-            int64_t ldy, const int32_t* idx, bool allow_split = true, bool pre_zeroed = false) {
+            int64_t ldy, const int32_t* idx, bool allow_split = true, bool pre_zeroed = false,
+            const tc::NextWeights* nx = nullptr) {
     if (use_tc) {
         const int epi = out_mode == 1 ? tc::kEpiScatterAtomic : (allow_split ? tc::kEpiAtomic : tc::kEpiStore);
-        return launch_gemm_tc(c, st, *tm, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed);
+        return launch_gemm_tc(c, st, *tm, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed, nullptr, nullptr,
+                              nullptr, nx);
     }
     if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx);
     return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
@@ -522,6 +597,12 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const int gemv_max = c->max_gemv_rows >= 0 ? c->max_gemv_rows : 0;
     auto tc_for = [&](int m) { return kBf16 && c->tc_ready && m > gemv_max; };
     int rc;
+    if (c->stamp_on && c->stamps) {  // fresh timing slots for this step: starts at the largest value, ends at zero
+        c->stamp_n = 0;
+        c->stamp_cls.clear();
+        CU_TRY(cudaMemsetAsync(c->stamps, 0xff, sizeof(uint64_t) * kStampCap, st));
+        CU_TRY(cudaMemsetAsync(c->stamps + kStampCap, 0, sizeof(uint64_t) * kStampCap, st));
+    }
     c->pdl_next = false;  // the first kernel of a step has no predecessor to overlap
     if ((rc = launch_k(c, st, kClsStepBegin, step_begin<WT>, dim3(B), dim3(256), 0, tokens,
                        static_cast<const WT*>(c->embed), D, V, kv->pos, c->inv_freq, hd / 2, c->x, c->cs, c->flags)))
@@ -555,6 +636,26 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool zero_qkv = t;  // (cleared even when a projection ends up with one K range and plain stores)
         const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
         const bool zero_gu = t && !fused_ffn;
+        // What each kernel of this layer asks the memory system to fetch for the projection after it (tensor-core
+        // path only): QKV -> all of W_o; attention -> the head of W_gate_up; gate/up -> the head of W_down;
+        // down -> the head of the next active layer's W_qkv (or of lm_head).
+        tc::NextWeights nx_o{}, nx_gu{}, nx_down{}, nx_after{};
+        if (t && (c->pf_depth > 0 || c->pf_attn_depth > 0 || c->pf_o) && !ph) {
+            nx_o = next_weights(c, &c->tm_wo[l], nullptr, D, c->qd, m, tc::kEpiScatterAtomic, c->pf_o ? (1 << 20) : 0);
+            if (fused_ffn)
+                nx_gu = next_weights(c, &c->tm_wgu[l], &c->tm_wgu64[l], F, D, m, tc::kEpiSwiglu, c->pf_attn_depth);
+            else
+                nx_gu = next_weights(c, &c->tm_wgu[l], nullptr, 2 * F, D, m, tc::kEpiAtomic, c->pf_attn_depth);
+            nx_down = next_weights(c, &c->tm_wd[l], nullptr, D, F, m, tc::kEpiScatterAtomic, c->pf_depth);
+            int ln = l + 1;
+            while (ln < L && c->cnt_h[ln] == 0) ++ln;
+            if (ln < L) {
+                if (tc_for(c->cnt_h[ln]))
+                    nx_after = next_weights(c, &c->tm_wqkv[ln], nullptr, c->qkvd, D, c->cnt_h[ln], tc::kEpiAtomic, c->pf_depth);
+            } else if (tc_for(B) && (logits || next_tokens)) {
+                nx_after = next_weights(c, &c->tm_lm, nullptr, V, D, B, tc::kEpiStore, c->pf_depth);
+            }
+        }
         // ---- attention half
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, static_cast<int32_t*>(nullptr),
@@ -567,7 +668,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                            route_here ? ph->tokscore + (size_t)l * ph->stride + ph->g0 : nullptr)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
-                              c->qkv, c->qkvd, nullptr, true, zero_qkv)))
+                              c->qkv, c->qkvd, nullptr, true, zero_qkv, &nx_o)))
             return rc;
         // The tuned attention kernel rotates q itself and appends the new token's key and value (its
         // row facts come from the norm kernel above); the general path has a kernel for that.
@@ -579,7 +680,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             return rc;
         if (mma_attn) {
             if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], &lkv, len_l, idx, t ? nullptr : c->att, xh, xl,
-                                      fuse_rope, qscale, pair_rows)))
+                                      fuse_rope, qscale, pair_rows, &nx_gu)))
                 return rc;
         } else {
             if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], &lkv, len_l, idx))) return rc;
@@ -598,11 +699,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
             if ((rc = launch_gemm_tc(c, st, c->tm_wgu64[l], c->tm_wgu[l], F, D, c->xh, c->xl, m, tc::kEpiSwiglu, nullptr, 0, nullptr,
-                                     false, nullptr, c->acth, c->actl)))
+                                     false, nullptr, c->acth, c->actl, &nx_down)))
                 return rc;
         } else {
             if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl,
-                                  m, 0, c->gu, 2 * F, nullptr, true, zero_gu)))
+                                  m, 0, c->gu, 2 * F, nullptr, true, zero_gu, &nx_down)))
                 return rc;
             if ((rc = launch_k(c, st, kClsSiluMul, silu_mul, dim3(std::min((m * F + 255) / 256, c->n_sm * 8)),
                                dim3(256), 0, c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr,
@@ -610,7 +711,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                 return rc;
         }
         if ((rc = project<WT>(c, st, t, c->w_down[l], t ? &c->tm_wd[l] : nullptr, D, F, c->act, c->acth, c->actl, m, 1,
-                              c->x, D, idx)))
+                              c->x, D, idx, true, false, &nx_after)))
             return rc;
     }
     if (ph) return FIRST_OK;  // a prefill chunk ends here: logits are taken once, from the last prompt tokens
@@ -749,7 +850,8 @@ int first_destroy(first_ctx* c) {
     if (!c) return FIRST_OK;
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
                     c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket, c->rowinfo,
-                    c->pf_cu, c->pf_tok, c->pf_cap, c->pf_pos, c->pf_len, c->pf_off, c->pf_ones, c->x_last, c->pf_score};
+                    c->pf_cu, c->pf_tok, c->pf_cap, c->pf_pos, c->pf_len, c->pf_off, c->pf_ones, c->x_last, c->pf_score,
+                    c->stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -998,7 +1100,27 @@ int first_last_device_flags(first_ctx* c, uint32_t* flags, void* stream) {
     CU_TRY(cudaMemcpyAsync(flags, c->flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaMemsetAsync(c->flags, 0, sizeof(uint32_t), st));
     CU_TRY(cudaStreamSynchronize(st));
+    if (*flags & FIRST_FLAG_WAIT_EXPIRED) {
+        // A kernel gave up on a wait: the step's outputs are undefined, and an attention work item that left
+        // early took no merge ticket.  Put the ticket counters back to zero so that later steps merge correctly.
+        CU_TRY(cudaMemsetAsync(c->ticket, 0, (size_t)c->d.max_batch * c->d.n_kv_heads * sizeof(uint32_t), st));
+        CU_TRY(cudaStreamSynchronize(st));
+    }
     return *flags ? FIRST_E_DEVICE_FLAG : FIRST_OK;
+}
+
+int first_selftest_wait_expiry(first_ctx* c, int32_t polls, int32_t* returned, int32_t* abort_word, void* stream) {
+    if (!c || polls <= 0 || polls > (1 << 20) || !returned || !abort_word) return FIRST_E_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* out = reinterpret_cast<int32_t*>(c->rowinfo);  // 16 bytes of scratch nothing else uses between steps
+    tc::wait_expiry_selftest<<<1, 32, 0, st>>>((uint32_t)polls, c->flags, out);
+    CU_TRY(cudaGetLastError());
+    int32_t h[2] = {-1, -1};
+    CU_TRY(cudaMemcpyAsync(h, out, sizeof h, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    *returned = h[0];
+    *abort_word = h[1];
+    return FIRST_OK;
 }
 
 int64_t first_launch_count(const first_ctx* c) { return c ? c->launches : 0; }
@@ -1049,8 +1171,23 @@ int first_sample_topk(const float* logits, int32_t B, int32_t vocab, int32_t top
     const bool greedy = top_k == 1 || temperature == 0.f;
     step_end_sample<<<B, 1024, 0, static_cast<cudaStream_t>(stream)>>>(logits, vocab, greedy ? 1 : top_k,
                                                                         greedy ? 1.f : 1.f / temperature, uniforms, tokens,
-                                                                        nullptr);
+                                                                        nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? FIRST_OK : FIRST_E_CUDA;
+}
+
+int first_step_trace(first_ctx* c, int32_t max_n, int32_t* cls, uint64_t* t_start, uint64_t* t_end, int32_t* n_out,
+                     void* stream) {
+    if (!c || !cls || !t_start || !t_end || !n_out || max_n < 0) return FIRST_E_ARG;
+    *n_out = 0;
+    if (!c->stamp_on || !c->stamps) return FIRST_E_STATE;
+    const int n = std::min<int>(c->stamp_n, max_n);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU_TRY(cudaMemcpyAsync(t_start, c->stamps, sizeof(uint64_t) * n, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaMemcpyAsync(t_end, c->stamps + kStampCap, sizeof(uint64_t) * n, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < n; ++i) cls[i] = c->stamp_cls[i];
+    *n_out = n;
+    return FIRST_OK;
 }
 
 int32_t first_kernel_class_count(void) { return kNumClasses; }
@@ -1072,6 +1209,16 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
+    else if (!std::strcmp(name, "pf_depth")) c->pf_depth = value >= 0 ? (int)value : 0;
+    else if (!std::strcmp(name, "pf_attn_depth")) c->pf_attn_depth = value >= 0 ? (int)value : 0;
+    else if (!std::strcmp(name, "pf_o")) c->pf_o = value > 0;
+    else if (!std::strcmp(name, "stamp")) {
+        c->stamp_on = value > 0;
+        if (c->stamp_on && !c->stamps) {
+            int rc = dev_alloc(&c->stamps, (size_t)2 * kStampCap);
+            if (rc) { c->stamp_on = 0; return rc; }
+        }
+    }
     else return FIRST_E_ARG;
     c->plan_version += 1;  // cached step graphs were built under the old options
     return FIRST_OK;

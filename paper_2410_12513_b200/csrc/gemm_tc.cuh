@@ -50,7 +50,43 @@ struct GemmParams {
     float* act;              // [m][n_out] float32 or NULL
     __nv_bfloat16* act_hi;   // [m][n_out] bfloat16 hi/lo split or NULL
     __nv_bfloat16* act_lo;
+    uint64_t* stamp;         // in-step timing slot or NULL
 };
+
+// What the NEXT weight-streaming kernel of the step will read first.  A kernel that has finished asking for
+// its own tiles (and so leaves HBM idle during its epilogue, the kernel boundary and the next kernel's
+// start-up) asks the memory system to bring the first `depth` k-blocks of every work unit of the next
+// projection into L2; that projection then starts on L2 hits.  The work units are enumerated exactly as
+// gemm_tc_kernel enumerates them.  mode 0: nothing; 1: tiles of mt x 128 rows; 2: gate|up pairs (two boxes
+// of `rows` rows, the second n_out rows further down).  A prefetch has no architectural effect: a wrong
+// guess costs bandwidth, never correctness.
+struct NextWeights {
+    CUtensorMap map;
+    int mode, tiles, ksplit, kblocks, depth, rows, n_out, mt;
+};
+
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
+
+// Called by ONE thread of CTA `cta` of `n_cta`: that CTA's share of the next projection's work units.
+__device__ __forceinline__ void prefetch_next_weights(const NextWeights& nx, int cta, int n_cta) {
+    if (nx.mode == 0) return;
+    const int units = nx.tiles * nx.ksplit;
+    for (int u = cta; u < units; u += n_cta) {
+        const int tile = u / nx.ksplit, split = u - tile * nx.ksplit;
+        const int kb0 = (int)((int64_t)nx.kblocks * split / nx.ksplit);
+        const int kb1 = min((int)((int64_t)nx.kblocks * (split + 1) / nx.ksplit), kb0 + nx.depth);
+        for (int kb = kb0; kb < kb1; ++kb) {
+            if (nx.mode == 2) {
+                tma_prefetch_2d(&nx.map, kb * kBlockK, tile * nx.rows);
+                tma_prefetch_2d(&nx.map, kb * kBlockK, nx.n_out + tile * nx.rows);
+            } else {
+                for (int a = 0; a < nx.mt; ++a) tma_prefetch_2d(&nx.map, kb * kBlockK, (tile * nx.mt + a) * kBlockM);
+            }
+        }
+    }
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -69,8 +105,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up after kSpinLimit polls (or when another role already gave up),
 // raising the CTA's abort word and the device flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_s, uint32_t* flags) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_s, uint32_t* flags,
+                                          uint32_t limit = kSpinLimit) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_s) return false;
     }
@@ -130,7 +167,9 @@ template <int EPI>
 __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                       const __grid_constant__ CUtensorMap tmA2,
                                                       const __grid_constant__ CUtensorMap tmBh,
-                                                      const __grid_constant__ CUtensorMap tmBl, const GemmParams p) {
+                                                      const __grid_constant__ CUtensorMap tmBl,
+                                                      const __grid_constant__ NextWeights nx, const GemmParams p) {
+    const Stamp stamp_guard(p.stamp);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int b_bytes = p.n_pad * 128;
@@ -215,12 +254,16 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
                 tma_load_2d(sa + a_bytes, &tmBh, full_bar(s), kc, 0);
                 if (p.use_lo) tma_load_2d(sa + a_bytes + b_bytes, &tmBl, full_bar(s), kc, 0);
             }
-            if (abort_s) {
-                // let the copies already issued land before this CTA's shared memory goes away
-                for (int i = max(0, issued - p.stages); i < issued; ++i) {
-                    const uint32_t bar = full_bar(i % p.stages), ph = (uint32_t)(i / p.stages) & 1u;
-                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, ph); ++it) {}
-                }
+            // every weight tile of this CTA has been asked for: from here on it leaves HBM idle
+            if (!abort_s) prefetch_next_weights(nx, (int)blockIdx.x, (int)gridDim.x);
+            // This lane does not reach the CTA's final barrier before every copy it issued has landed (the last
+            // use of each stage; earlier uses were consumed before their stage was refilled).  It does so
+            // whether or not any role has given up and whichever role notices first: the CTA's shared memory
+            // can therefore never be handed to another CTA with a copy still in flight.  In a normal run the
+            // consumers wait for the same barriers anyway, so this costs nothing.
+            for (int i = max(0, issued - p.stages); i < issued; ++i) {
+                const uint32_t bar = full_bar(i % p.stages), ph = (uint32_t)(i / p.stages) & 1u;
+                for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, ph); ++it) {}
             }
         }
     } else if (warp == 1) {
@@ -356,8 +399,30 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
+        // After a failed wait the epilogue may have left without seeing the accumulator complete: the MMAs that
+        // were issued (their operands had landed, so they finish) must be done before the tensor memory and the
+        // shared memory they use are given back.  The commit above arrives on this barrier once they are.
+        if (abort_s && lane == 0)
+            for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(tmem_full_bar, 0u); ++it) {}
+        __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)p.tmem_cols)
                      : "memory");
+    }
+}
+
+// Exercises the give-up path of mbar_wait without any copy in flight: a barrier that expects one arrival
+// which never comes.  The wait runs out after `limit` polls, raises the abort word and the device flag, and
+// the kernel returns normally.  out[0] = what the wait returned, out[1] = the abort word.
+static __global__ void wait_expiry_selftest(uint32_t limit, uint32_t* flags, int32_t* out) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_s;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_s, flags, limit);
+        out[0] = ok ? 1 : 0;
+        out[1] = abort_s;
     }
 }
 

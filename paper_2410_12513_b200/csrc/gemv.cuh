@@ -16,7 +16,9 @@ enum GemvEpilogue { kStore = 0, kScatterAdd = 1 };
 template <typename WT, int R, int EPI>
 __global__ void __launch_bounds__(256) gemv_rows(const WT* __restrict__ W, int n_out, int K,
                                                  const float* X, int r0, int rows_valid,
-                                                 float* __restrict__ Y, int64_t ldy, const int32_t* __restrict__ idx) {
+                                                 float* __restrict__ Y, int64_t ldy, const int32_t* __restrict__ idx,
+                                                 uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const int lane = threadIdx.x & 31;

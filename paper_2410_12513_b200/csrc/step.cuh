@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(256) step_begin(const int32_t* __restrict__ to
                                                   int D, int V, const int32_t* __restrict__ pos,
                                                   const double* __restrict__ inv_freq, int half,
                                                   float* __restrict__ x, float2* __restrict__ cs,
-                                                  uint32_t* __restrict__ flags) {
+                                                  uint32_t* __restrict__ flags, uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const int b = blockIdx.x;
@@ -75,7 +76,8 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
                                                      uint32_t* __restrict__ flags,
                                                      const float* __restrict__ router_w,
                                                      const float* __restrict__ router_b, int router_mode,
-                                                     float* __restrict__ tok_out) {
+                                                     float* __restrict__ tok_out, uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     // One pass: the row stays in registers between the sum of squares and the scaling
     // (up to kMaxV float4 per thread; longer rows re-read the tail from L1/L2).
     constexpr int kMaxV = 4;
@@ -174,7 +176,8 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                                                   const int64_t* __restrict__ slab_off,
                                                   const int32_t* __restrict__ slab_cap,
                                                   const int32_t* len_l, uint32_t* __restrict__ flags,
-                                                  longlong2* __restrict__ rowinfo, int pair) {
+                                                  longlong2* __restrict__ rowinfo, int pair, uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const int i = blockIdx.y, head = blockIdx.x * blockDim.y + threadIdx.y, d = threadIdx.x, b = idx[i];
@@ -228,7 +231,9 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
 
 // act[i][f] = silu(gate) * up from gu[i] = [gate(F) | up(F)]; optional bf16 hi/lo split.
 __global__ void __launch_bounds__(256) silu_mul(const float* gu, int m, int F, float* __restrict__ act,
-                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const size_t n = (size_t)m * F;
@@ -248,7 +253,8 @@ __global__ void __launch_bounds__(256) silu_mul(const float* gu, int m, int F, f
 // End of a step: greedy next token per row (lowest index among equal maxima) and pos += 1.
 // One block of 1024 threads per row; 16-byte loads when the row allows it.
 __global__ void __launch_bounds__(1024) step_end(const float* logits, int V, int32_t* __restrict__ next,
-                                                 int32_t* __restrict__ pos) {
+                                                 int32_t* __restrict__ pos, uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const int b = blockIdx.x;
@@ -307,7 +313,9 @@ __device__ __forceinline__ bool sample_before(float v, int i, float w, int j) { 
 
 __global__ void __launch_bounds__(1024) step_end_sample(const float* logits, int V, int k, float inv_T,
                                                         const float* __restrict__ uniforms,
-                                                        int32_t* __restrict__ next, int32_t* __restrict__ pos) {
+                                                        int32_t* __restrict__ next, int32_t* __restrict__ pos,
+                                                        uint64_t* stamp) {
+    const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
     const int b = blockIdx.x;

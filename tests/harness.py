@@ -9,12 +9,7 @@ import oracle
 
 
 # ------------------------------------------------------------------ oracle side
-def oracle_model(shape, weights, kv_bf16=None):
-    return oracle.OracleModel(oracle.Shape(**shape.asdict()), weights, kv_bf16)
-
-
-def widen(a):
-    return fi.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a
+from oracle.workload import oracle_model, stand_in_cache, widen  # noqa: E402,F401
 
 
 # ------------------------------------------------------------------ CUDA side
@@ -97,34 +92,21 @@ class GpuKV:
 def synthetic_caches(shape, lens, caps, seed, bf16, layers=None, with_gpu=True):
     """Stand-in prefilled caches N(0,1) for every (layer, sequence): identical values on both
     sides.  lens: [B] tokens present in every layer; pos = lens."""
-    B, L = len(lens), shape.n_layers
-    okv = oracle.OracleKV(oracle.Shape(**shape.asdict()), caps)
     gkv = GpuKV(shape, caps, bf16, layers) if with_gpu else None
-    layers = range(L) if layers is None else layers
-    for l in layers:
-        for b in range(B):
-            n = int(lens[b])
-            kr = fi.synthetic_kv_rows(n, shape.kv_dim, seed, f"k{l}_{b}", bf16)
-            vr = fi.synthetic_kv_rows(n, shape.kv_dim, seed, f"v{l}_{b}", bf16)
-            ko, vo = okv.rows(l, b)
-            ko[:n] = widen(kr)
-            vo[:n] = widen(vr)
-            if gkv is not None:
-                gkv.load_rows(l, b, kr, vr)
-    okv.len[:] = np.asarray(lens, dtype=np.int32)[None, :]
-    okv.pos[:] = np.asarray(lens, dtype=np.int32)
+    okv = stand_in_cache(shape, lens, caps, seed, bf16, layers, sink=gkv.load_rows if gkv is not None else None)
     if gkv is not None:
         gkv.set_len(okv.len, okv.pos)
     return okv, gkv
 
 
 # ------------------------------------------------------------------ router calibration
-def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3, tight=False):
+def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3, tight=False, bias=None):
     """Router weights w[D] (no bias) that realise `target_keep` on the given per-sequence hidden
     states with every oracle score at least `margin` away from tau.  Least-norm solve on the
     pooled means (B <= D), scaled up until the oracle's own scores clear the margin.
     tight=True: scaled so that the score nearest to tau lies in [margin, 2*margin] -- the stated
-    margin itself, not a comfortable multiple of it."""
+    margin itself, not a comfortable multiple of it.  bias: a fixed router bias (for tau != 0.5 the
+    bias logit(tau) centres the scores on tau, which a bias-free router cannot do near the margin)."""
     B = len(hiddens)
     pooled = np.stack([h.astype(np.float64).mean(0) for h in hiddens])  # [B][D]
     t = np.where(np.asarray(target_keep) > 0, 1.0, -1.0)
@@ -135,7 +117,7 @@ def calibrate_router(hiddens, target_keep, mode, seed, tau=0.5, margin=1e-3, tig
 
     def scores(c):
         w = (pinv @ (c * t * spread)).astype(np.float32)
-        rho = np.array([oracle.route(h, w, None, tau, mode)[0] for h in hiddens])
+        rho = np.array([oracle.route(h, w, bias, tau, mode)[0] for h in hiddens])
         return w, rho
 
     if tight:

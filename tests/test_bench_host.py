@@ -75,3 +75,43 @@ def test_replica_aggregation_over_two_gloo_ranks():
     assert res == {0: 125.0, 1: 125.0}       # both ranks agree on the slowest time
     assert bench.job_tokens_per_s(2, 32, 10, 125.0) == 2 * 32 * 10 / 0.125
     assert bench.max_over_ranks(7.5, None, None) == 7.5
+
+
+_STUB = '''
+import json, os, sys
+sys.path.insert(0, {root!r})
+import torch
+import torch.distributed as dist
+import bench
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+assert os.environ["FIRST_BENCH_BACKEND"] == "gloo" and os.environ["LOCAL_RANK"] == "0"
+dist.init_process_group("gloo")                      # MASTER_ADDR / MASTER_PORT from the spawner
+ms = bench.max_over_ranks(100.0 + 25.0 * rank, dist, torch.device("cpu"))
+dist.barrier()
+rec = dict(rank=rank, world=world, gpu=os.environ["CUDA_VISIBLE_DEVICES"], ms=ms, argv=sys.argv[1:],
+           addr=os.environ["MASTER_ADDR"])
+open(os.path.join({out!r}, f"rank{{rank}}.json"), "w").write(json.dumps(rec))
+if rank == 0:
+    print(json.dumps(dict(n_gpus=world, value=bench.job_tokens_per_s(world, 32, 10, ms))))
+dist.destroy_process_group()
+sys.exit(3 if (rank == 1 and "--fail" in sys.argv) else 0)
+'''
+
+
+def test_gpus_n_starts_n_replicas_one_process_per_gpu(tmp_path, capfd):
+    """`bench.py --gpus N` outside torchrun starts the N replicas itself: replica i gets GPU i alone, rank i of N,
+    a 127.0.0.1 rendezvous; rank 0's line is passed through; the slowest replica's time is what all agree on.
+    A stub stands in for the GPU work (gloo, 2 ranks)."""
+    import json
+    stub = tmp_path / "stub_worker.py"
+    stub.write_text(_STUB.format(root=str(ROOT), out=str(tmp_path)))
+    rc = bench.spawn_replicas(2, ["--steps", "10"], script=[str(stub)], timeout=300)
+    assert rc == 0
+    recs = [json.loads((tmp_path / f"rank{r}.json").read_text()) for r in range(2)]
+    assert [r["gpu"] for r in recs] == ["0", "1"] and [r["rank"] for r in recs] == [0, 1]
+    assert all(r["world"] == 2 and r["ms"] == 125.0 and r["argv"] == ["--steps", "10"] and r["addr"] == "127.0.0.1"
+               for r in recs)
+    line = json.loads(capfd.readouterr().out.strip().splitlines()[-1])
+    assert line == {"n_gpus": 2, "value": 2 * 32 * 10 / 0.125}
+    # a failing replica fails the job
+    assert bench.spawn_replicas(2, ["--fail"], script=[str(stub)], timeout=300) == 3

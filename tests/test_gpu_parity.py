@@ -76,12 +76,14 @@ def test_router_masks_bit_exact_at_the_stated_margin(hidden_bf16, mode):
         hs = [hid_f[cu[b]:cu[b + 1]] for b in range(B)]
         target = fi.mask_bernoulli(B, 3, 0.5, 200 + l)[:, 1]
         tau = 0.5 if l < 3 else 0.4
-        rw, _ = calibrate_router(hs, target, mode, l, tau=tau, tight=True)
-        want_rho[:, l], want_mask[:, l] = oracle.route_batch(hid_f, cu, rw, None, tau, mode)
+        bias = None if l < 3 else float(np.log(tau / (1.0 - tau)))  # centres the scores on tau
+        rw, _ = calibrate_router(hs, target, mode, l, tau=tau, tight=True, bias=bias)
+        want_rho[:, l], want_mask[:, l] = oracle.route_batch(hid_f, cu, rw, bias, tau, mode)
         gap = np.abs(want_rho[:, l] - tau)
         assert 1e-3 <= gap.min() <= 2e-3 and gap.max() <= 2.5e-3, gap
         assert np.array_equal(want_mask[:, l], target)
-        args = (to_dev(hid, hidden_bf16), torch.from_numpy(cu).cuda(), to_dev(rw, False), None, tau, mode)
+        b_t = None if bias is None else torch.tensor([bias], dtype=torch.float32, device="cuda")
+        args = (to_dev(hid, hidden_bf16), torch.from_numpy(cu).cuda(), to_dev(rw, False), b_t, tau, mode)
         ctx.prefill_route(l, *args, mask, scores)
         first_prefill_route_static(l, L, *args, mask_s, None, flags)
     assert ctx.device_flags() == 0 and int(flags.item()) == 0
@@ -406,6 +408,31 @@ def test_full_slab_on_the_tuned_attention_path():
     ref = oracle.decode_step(om, toks[1:2], np.ones((1, shape.n_layers), np.uint8), solo)
     err, _ = logits_check(logits[1:2].cpu().numpy(), ref)
     assert err.max() <= 2e-2
+
+
+def test_a_wait_that_runs_out_raises_the_flag_and_the_context_stays_usable():
+    """The give-up path of the kernels' bounded waits, made to run out on purpose (a barrier nothing completes,
+    no copy in flight): the kernel returns, the abort word and FIRST_FLAG_WAIT_EXPIRED are set, and the same
+    context then decodes correctly."""
+    import torch
+    shape = fi.TINY
+    errs, _ = _run_decode_case(shape, False, [5, 9], np.ones((2, shape.n_layers), np.uint8), 1, 8, 1e-4)
+    from paper_2410_12513_b200 import FirstContext
+    w = fi.make_weights(shape, 8, False)
+    ctx = _ctx(shape, False, 2, 16, w)
+    assert ctx.selftest_wait_expiry(1000) == (0, 1)
+    assert ctx.device_flags() == 8
+    assert ctx.device_flags() == 0
+    # still good for a step
+    om = oracle_model(shape, w)
+    okv, gkv = synthetic_caches(shape, [5, 9], [8, 12], 8, False)
+    mask = np.ones((2, shape.n_layers), np.uint8)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = fi.tokens(shape, 2, 8, "first")
+    logits = torch.empty((2, shape.vocab), dtype=torch.float32, device="cuda")
+    ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits)
+    err, _ = logits_check(logits.cpu().numpy(), oracle.decode_step(om, toks, mask, okv))
+    assert err.max() <= 1e-4 and ctx.device_flags() == 0
 
 
 def test_bad_token_sets_flag():
