@@ -31,8 +31,8 @@
  *     first_destroy; the two later allocations are stated where they happen (first_prefill's
  *     token scores, the internal logits row buffer of first_decode_step without `logits`).
  *   - Work is enqueued on the CUDA stream passed as `void *stream` (a cudaStream_t;
- *     NULL = the default stream).  Only first_set_mask and first_last_device_flags
- *     wait for the stream.
+ *     NULL = the default stream).  Only first_set_mask, first_prefill, first_last_device_flags
+ *     and the measurement aids wait for the stream.
  *   - Layers are numbered from 0.  mask[b][l] is a byte, 1 = sequence b runs layer l,
  *     0 = it skips it.  All matrices are row-major; linear weights are [out][in].
  *   - dtype FIRST_DTYPE_F32: weight matrices and KV cache are float32.
@@ -240,6 +240,16 @@ int first_prefill(first_ctx *ctx, const int32_t *tokens, const int32_t *cu_seqle
  * other than 0/1), FIRST_E_CUDA. */
 int first_set_mask(first_ctx *ctx, const uint8_t *mask, int32_t B, void *stream);
 
+/* first_set_mask for a mask held in HOST memory, without waiting for the stream (a batch that changes
+ * between steps should not stall the device: decisions are per sequence and fixed for its whole decode,
+ * "Inference for FiRST" item 2, so sequences come and go independently).  The per-layer counts are taken
+ * on the host; the launches of later steps are sized from them rounded up to a multiple of 16 and the
+ * kernels read the exact counts from device memory, so a recorded step graph is found again after any
+ * change of the batch that leaves every layer's count inside its bucket of 16.
+ *   mask  host uint8 [B][n_layers], bytes 0/1 (FIRST_E_ARG otherwise); copied before the call returns
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_STATE (stream being captured), FIRST_E_CUDA. */
+int first_set_mask_host(first_ctx *ctx, const uint8_t *mask, int32_t B, void *stream);
+
 /* Read back the plan of the last first_set_mask (for inspection and tests).
  *   idx   host int32 [n_layers][B]: idx[l][0..cnt[l]-1] ascending active rows, rest -1
  *   cnt   host int32 [n_layers]
@@ -265,6 +275,51 @@ int first_get_plan(first_ctx *ctx, int32_t *idx, int32_t *cnt, int32_t *slot);
  * slab or a bad token id. */
 int first_decode_step(first_ctx *ctx, const int32_t *tokens, const first_kv_cache *kv, float *logits,
                       int32_t *next_tokens, float *layer_inputs, void *stream);
+
+/* Batches whose membership changes between steps ("Inference for FiRST", item 2: a sequence's layer
+ * decisions are fixed once its prompt has been routed, and a layer it skips needs no cache).  A pool
+ * manages row ranges ("slabs") of caller-owned per-layer cache tensors: a sequence that joins gets a
+ * batch row (slot) and, in every layer it KEEPS, a slab of `capacity` token rows; layers it skips get
+ * nothing, so the cache memory in use is the sum over kept (sequence, layer) pairs.  The pool keeps the
+ * per-layer slab tables of first_kv_cache (per_layer = 1) in device memory and its sequences' masks on
+ * the host.  None of these calls waits for the stream; all calls of a pool, and the decode steps on its
+ * cache, belong on one stream (a slab freed by first_seq_leave may be handed out by the next join).
+ *
+ * first_pool_create   max_seqs <= max_batch batch rows; rows_per_layer host int64 [L]: token rows of layer
+ *                     l's tensors k[l], v[l] (dev [Hkv][rows_per_layer[l]][hd], caller-owned, borrowed for
+ *                     the pool's lifetime).  Allocates the pool's small device tables.
+ * first_seq_join      mask_row host uint8 [L] (the sequence's decisions); capacity = slab rows per kept layer
+ *                     (<= max_tokens_per_seq).  src != NULL: the keys/values of the sequence's first
+ *                     n_tokens tokens are copied, for the kept layers, from sequence src_seq of cache `src`
+ *                     (per_layer = 0, e.g. the cache a first_prefill call filled), len = pos = n_tokens;
+ *                     src == NULL: empty slabs, n_tokens must be 0.  *slot = the batch row: the caller
+ *                     feeds the sequence's tokens at tokens[slot] and reads its logits at row slot.
+ *                     FIRST_E_CAPACITY: no free batch row, or some kept layer has no free range of
+ *                     `capacity` rows (nothing is taken then).
+ * first_seq_leave     frees the slot and its slabs.
+ * first_pool_commit   rebuilds the step's per-layer active-row plan for the sequences now in the pool
+ *                     (first_set_mask_host over all max_seqs batch rows; free rows skip every layer).  Call
+ *                     after a group of joins and leaves, before the next first_decode_step.
+ * first_pool_kv       fills *out with the pool's cache view (per_layer = 1) for first_decode_step; tokens
+ *                     and outputs of a step have max_seqs rows; free rows need a valid token id.
+ * first_pool_stats    rows_held[l] = token rows handed out in layer l, largest_free[l] = longest free range,
+ *                     *live = sequences in the pool (host arrays of L entries, any may be NULL).
+ * Errors: FIRST_E_ARG, FIRST_E_CAPACITY, FIRST_E_UNSUPPORTED (more than 96 layers), FIRST_E_STATE (leave of
+ * a free slot), FIRST_E_CUDA. */
+typedef struct first_pool first_pool;
+int first_pool_create(first_ctx *ctx, int32_t max_seqs, const int64_t *rows_per_layer, void *const *k, void *const *v,
+                      first_pool **out);
+int first_pool_destroy(first_pool *pool);
+int first_seq_join(first_pool *pool, const uint8_t *mask_row, int32_t capacity, const first_kv_cache *src,
+                   int32_t src_seq, int32_t n_tokens, int32_t *slot, void *stream);
+int first_seq_leave(first_pool *pool, int32_t slot, void *stream);
+int first_pool_commit(first_pool *pool, void *stream);
+int first_pool_kv(first_pool *pool, first_kv_cache *out);
+int first_pool_stats(first_pool *pool, int64_t *rows_held, int64_t *largest_free, int32_t *live);
+
+/* The description a context was created with; the number of recorded step graphs it holds. */
+int first_get_desc(const first_ctx *ctx, first_model_desc *out);
+int64_t first_graph_count(const first_ctx *ctx);
 
 /* Next-token sampling with the paper's generation settings (appendix "Training and Inference
  * Setup", inference settings: temperature 0.8, top-k sampling over 10 tokens).  Per row: the
@@ -337,8 +392,9 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *   "tc_use_lo"      0 = tensor-core projections use only the bfloat16 hi half of activations
  *   "use_graph"      0 = launch every kernel of a step directly.  Default 1: first_decode_step
  *                    records its launch sequence once per distinct set of pointer arguments
- *                    (tokens, outputs, cache tensors) and plan, as a CUDA graph, and
- *                    replays it; up to 8 such graphs are kept.  Nothing is captured while the
+ *                    (tokens, outputs, cache tensors) and per-layer launch rows, as a CUDA graph, and
+ *                    replays it; up to 16 such graphs are kept (least recently used dropped), across
+ *                    first_set_mask calls: the row lists live in device memory, not in the graph.  Nothing is captured while the
  *                    caller's stream is itself being captured or while first_profile is on.
  *   "tc_lo_max_rows" the hi/lo activation split is used for projections with at most this many
  *                    active rows, the hi half alone above (default: always both halves; the hi

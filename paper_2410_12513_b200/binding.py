@@ -86,6 +86,22 @@ def lib():
         L.first_profile.restype = C.c_int
         L.first_profile_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_profile_read.restype = C.c_int
+        L.first_set_mask_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.first_set_mask_host.restype = C.c_int
+        L.first_pool_create.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
+                                        C.POINTER(C.c_void_p)]
+        L.first_pool_destroy.argtypes = [C.c_void_p]
+        L.first_seq_join.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(KVCacheC), C.c_int32, C.c_int32,
+                                     C.POINTER(C.c_int32), C.c_void_p]
+        L.first_seq_leave.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.first_pool_commit.argtypes = [C.c_void_p, C.c_void_p]
+        L.first_pool_kv.argtypes = [C.c_void_p, C.POINTER(KVCacheC)]
+        L.first_pool_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+        for name in ("first_pool_create", "first_pool_destroy", "first_seq_join", "first_seq_leave", "first_pool_commit",
+                     "first_pool_kv", "first_pool_stats"):
+            getattr(L, name).restype = C.c_int
+        L.first_graph_count.argtypes = [C.c_void_p]
+        L.first_graph_count.restype = C.c_int64
         L.first_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.first_selftest_wait_expiry.restype = C.c_int
         L.first_step_trace.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -226,6 +242,87 @@ def first_set_mask(h, mask, stream=None):
         raise FirstError(rc, "first_set_mask")
 
 
+def first_set_mask_host(h, mask, stream=None):
+    """mask: HOST uint8 [B][L] (numpy or CPU tensor); no wait for the stream."""
+    import numpy as np
+    m = np.ascontiguousarray(np.asarray(mask), dtype=np.uint8)
+    rc = lib().first_set_mask_host(h, m.ctypes.data, m.shape[0], _stream(stream))
+    if rc:
+        raise FirstError(rc, "first_set_mask_host")
+
+
+class _PoolKV:
+    """The pool's cache view (a first_kv_cache with per-layer tables that live in the pool)."""
+
+    def __init__(self, c):
+        self.c = c
+
+
+class FirstPool:
+    """Slab pool over caller-owned per-layer cache tensors for batches that change between steps
+    (first_pool_* / first_seq_* in first.h).  k, v: lists of CUDA tensors [Hkv][rows_l][hd]."""
+
+    def __init__(self, ctx, max_seqs, k, v):
+        import numpy as np
+        self._k, self._v, self._ctx = k, v, ctx
+        self.L, self.B = len(k), int(max_seqs)
+        rows = np.array([0 if t is None else int(t.shape[1]) for t in k], dtype=np.int64)
+        first = next(t for t in k if t is not None)
+        ka, va = _ptr_array(k, first.dtype, "pool.k"), _ptr_array(v, first.dtype, "pool.v")
+        self.h = C.c_void_p()
+        rc = lib().first_pool_create(ctx.h, self.B, rows.ctypes.data, C.cast(ka, C.POINTER(C.c_void_p)),
+                                     C.cast(va, C.POINTER(C.c_void_p)), C.byref(self.h))
+        if rc:
+            raise FirstError(rc, "first_pool_create")
+        c = KVCacheC()
+        rc = lib().first_pool_kv(self.h, C.byref(c))
+        if rc:
+            raise FirstError(rc, "first_pool_kv")
+        self.kv = _PoolKV(c)
+
+    def close(self):
+        if self.h:
+            lib().first_pool_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def join(self, mask_row, capacity, src=None, src_seq=0, n_tokens=0, stream=None):
+        import numpy as np
+        m = np.ascontiguousarray(np.asarray(mask_row), dtype=np.uint8)
+        slot = C.c_int32(-1)
+        rc = lib().first_seq_join(self.h, m.ctypes.data, int(capacity), C.byref(src.c) if src is not None else None,
+                                  int(src_seq), int(n_tokens), C.byref(slot), _stream(stream))
+        if rc:
+            raise FirstError(rc, "first_seq_join")
+        return slot.value
+
+    def leave(self, slot, stream=None):
+        rc = lib().first_seq_leave(self.h, int(slot), _stream(stream))
+        if rc:
+            raise FirstError(rc, "first_seq_leave")
+
+    def commit(self, stream=None):
+        rc = lib().first_pool_commit(self.h, _stream(stream))
+        if rc:
+            raise FirstError(rc, "first_pool_commit")
+        self._ctx.B = self.B
+
+    def stats(self):
+        import numpy as np
+        held = np.zeros(self.L, dtype=np.int64)
+        big = np.zeros(self.L, dtype=np.int64)
+        live = C.c_int32(0)
+        rc = lib().first_pool_stats(self.h, held.ctypes.data, big.ctypes.data, C.byref(live))
+        if rc:
+            raise FirstError(rc, "first_pool_stats")
+        return held, big, live.value
+
+
 def first_get_plan(h, B, L):
     import numpy as np
     idx = np.empty((L, B), dtype=np.int32)
@@ -342,6 +439,14 @@ class FirstContext:
     def set_mask(self, mask, stream=None):
         first_set_mask(self.h, mask, stream)
         self.B = mask.shape[0]
+
+    def set_mask_host(self, mask, stream=None):
+        import numpy as np
+        first_set_mask_host(self.h, mask, stream)
+        self.B = np.asarray(mask).shape[0]
+
+    def graph_count(self):
+        return int(lib().first_graph_count(self.h))
 
     def get_plan(self):
         return first_get_plan(self.h, self.B, self.shape.n_layers)

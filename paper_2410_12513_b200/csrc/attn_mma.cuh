@@ -78,13 +78,13 @@ template <int HD, int G, bool PAIR = false>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
                                                       const float* q, int64_t cap_total,
-                                                      const longlong2* rowinfo, int Hq, int C,
+                                                      const longlong2* rowinfo, const int32_t* __restrict__ m_dev,
+                                                      int Hq, int C,
                                                       float* __restrict__ o_part, float2* __restrict__ ml_part,
                                                       uint32_t* __restrict__ ticket, float* __restrict__ out,
                                                       __nv_bfloat16* __restrict__ out_hi,
                                                       __nv_bfloat16* __restrict__ out_lo,
                                                       uint32_t* __restrict__ flags, const RopeFuse rf,
-                                                      const __grid_constant__ tc::NextWeights nx,
                                                       uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     constexpr int kHalves = HD / 64;              // 128-byte column groups per row
@@ -95,6 +95,11 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     static_assert(GR <= 8, "query heads of a group (of two rows' groups) are the 8 hi rows of the A fragment");
 
     pdl_trigger();
+    // m_dev: the layer's active-row count (the grid is sized from a host-side upper bound of it)
+    if (m_dev && (int)blockIdx.z >= __ldg(m_dev)) {
+        pdl_wait();  // a grid must not complete before its predecessor has: later kernels rely on that chain
+        return;
+    }
     // Set-up that needs nothing from the previous kernel comes first, so that it overlaps that kernel's tail.
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -113,12 +118,6 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     }
     __syncthreads();
     pdl_wait();
-    if (threadIdx.x == 129) {
-        // This kernel is latency-bound and leaves about half of the HBM bandwidth unused: one thread per CTA
-        // (work items that turn out empty included) asks for the first weight tiles of the next projection.
-        const int cta = (int)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x);
-        tc::prefetch_next_weights(nx, cta, (int)(gridDim.x * gridDim.y * gridDim.z));
-    }
     const int S_max = gridDim.x, c = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     // (tokens to attend over incl. the new one | batch row << 32, first slab row | append << 62)
     const longlong2 ri = __ldcg(&rowinfo[i]);

@@ -16,12 +16,14 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
                                                          const int64_t* __restrict__ slab_off,
                                                          const int32_t* len_l,
                                                          const int32_t* __restrict__ slab_cap,
-                                                         const int32_t* __restrict__ idx, int Hq,
+                                                         const int32_t* __restrict__ idx,
+                                                         const int32_t* __restrict__ m_dev, int Hq,
                                                          float* __restrict__ o_part, float2* __restrict__ ml_part,
                                                          uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
+    if (m_dev && (int)blockIdx.z >= __ldg(m_dev)) return;  // beyond the layer's active rows (grid sized from a bound)
     constexpr int EPL = HD / 32;
     const int S = gridDim.x, s = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     const int b = idx[i];
@@ -97,12 +99,14 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
 // Merge the S partial results of each (row, query head): out[i][hq*HD + d] (float32) and,
 // optionally, its bfloat16 hi/lo split for the tensor-core O-projection.
 __global__ void __launch_bounds__(128) attn_combine(const float* o_part, const float2* ml_part,
+                                                    const int32_t* __restrict__ m_dev, int Hq,
                                                     int S, int HD, float* __restrict__ out,
                                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                     uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
+    if (m_dev && (int)(blockIdx.x / Hq) >= __ldg(m_dev)) return;
     const size_t hq = blockIdx.x;  // flat (row, query head)
     float M = -INFINITY;
     for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[hq * S + s].x);

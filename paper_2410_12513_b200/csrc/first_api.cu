@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "first.h"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "gemv.cuh"
 #include "prefill.cuh"
 #include "router.cuh"
@@ -84,7 +85,8 @@ struct first_ctx {
         uint64_t last_use = 0;
     };
     std::vector<StepGraph> graphs;
-    uint64_t plan_version = 0, use_clock = 0;
+    uint64_t plan_version = 0, use_clock = 0;  // plan_version: bumped by option and sampling changes
+    uint8_t* mask_dev = nullptr;               // [max_batch][L]: device copy of a mask given on the host
     cudaStream_t cap_stream = nullptr;  // steps are recorded here (the caller's stream may be the default one)
     int use_graph = 1;
     int use_pdl = 1;
@@ -95,9 +97,7 @@ struct first_ctx {
     int stamp_n = 0;
     std::vector<int> stamp_cls;
     // options
-    int pf_depth = 0;       // k-blocks per work unit of the next projection that a projection's idle producer prefetches
-    int pf_attn_depth = 0;  // the same for the attention kernel (head of the gate/up weights)
-    int pf_o = 0;           // the QKV projection prefetches the whole O matrix
+    int tc2_min_rows = 0;   // from this many rows on a projection launch uses the CTA-pair kernel (0 = never)
     int max_gemv_rows = -1;
     int attn_simple = -1;
     int tc_use_lo = 1;
@@ -305,41 +305,97 @@ TcShape tc_shape(const first_ctx* c, int n_out, int K, int mm, int epi) {
     return t;
 }
 
-// What the projection (weights tm / tm_pair, n_out x K, m rows, epilogue epi) will read first: handed to the
-// kernel that runs before it (see tc::NextWeights).  depth = k-blocks per work unit; 0 rows or depth: nothing.
-tc::NextWeights next_weights(const first_ctx* c, const CUtensorMap* tm, const CUtensorMap* tm_pair, int n_out, int K,
-                             int m, int epi, int depth) {
-    tc::NextWeights nx{};
-    if (!tm || m <= 0 || m > 256 || depth <= 0) return nx;
-    const TcShape t = tc_shape(c, n_out, K, m, epi);
-    const bool pairs = epi == tc::kEpiSwiglu;
-    nx.map = (pairs && t.mt == 1) ? *tm_pair : *tm;
-    nx.mode = pairs ? 2 : 1;
-    nx.tiles = t.tiles;
-    nx.ksplit = t.ksplit;
-    nx.kblocks = t.kblocks;
-    nx.depth = depth;
-    nx.rows = pairs ? t.tile_rows : tc::kBlockM;
-    nx.n_out = n_out;
-    nx.mt = t.mt;
-    if (pairs && t.mt == 2) {  // two 128-row boxes per half: gate rows tile*128.., up rows n_out + tile*128..
-        nx.rows = 128;
+// The CTA-pair kernel (gemm_tc2.cuh) for launches of many rows.  Units = (group of two 256-row weight tiles, K
+// range); the K ranges fill the SM pairs in whole waves.
+constexpr int kTc2SmemMax = 226 * 1024;
+
+bool tc2_wanted(const first_ctx* c, int mm, int n_out, int epi) {
+    if (c->tc2_min_rows <= 0 || mm < c->tc2_min_rows || mm > 256) return false;
+    if (epi == tc::kEpiSwiglu && n_out % 256) return false;
+    return true;
+}
+
+int launch_gemm_tc2(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n_out, int K, const __nv_bfloat16* Xh,
+                    const __nv_bfloat16* Xl, int mm, int r0, int epi, float* Y, int64_t ldy, const int32_t* idx,
+                    bool pre_zeroed, float* act, __nv_bfloat16* act_hi, __nv_bfloat16* act_lo, const int32_t* m_dev) {
+    int rc;
+    tc::GemmParams p{};
+    p.n_out = n_out; p.K = K; p.m = mm;
+    p.n_pad = (mm + 31) / 32 * 32;  // half of the activation rows in each CTA, in whole 16-row groups
+    p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
+    p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
+    p.mt = 2;
+    p.pair_rows = 0;
+    const int tiles = epi == tc::kEpiSwiglu ? (n_out + 255) / 256 : (n_out + 511) / 512;
+    const int stage_bytes = tc::kABytes * p.mt + (p.n_pad / 2) * 128 * (p.use_lo ? 2 : 1);
+    p.stages = std::max(2, std::min(8, (kTc2SmemMax - 2048) / stage_bytes));
+    p.ksplit = tc_ksplit(c, tiles, K, epi, mm, std::max(1, c->n_sm / 2));
+    int cols = 32;
+    while (cols < p.n_pad) cols *= 2;
+    p.acc_cols = cols;
+    p.tmem_cols = std::max(32, cols * p.mt);
+    p.act = act; p.act_hi = act_hi; p.act_lo = act_lo;
+    p.Y = Y; p.ldy = ldy; p.idx = idx;
+    p.flags = c->flags;
+    p.stamp = stamp_slot(c, kClsGemmTc);
+    p.m_dev = m_dev;
+    p.row0 = r0;
+    CUtensorMap tmBh, tmBl;
+    if ((rc = make_map(&tmBh, Xh, mm, K, p.n_pad / 2, false))) return rc;
+    if ((rc = make_map(&tmBl, Xl, mm, K, p.n_pad / 2, false))) return rc;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 8 * (2 * p.stages + 1) + 64;
+    int e = epi;
+    if (e == tc::kEpiAtomic) {
+        if (p.ksplit == 1) e = tc::kEpiStore;
+        else if (!pre_zeroed) {
+            CU_TRY(cudaMemsetAsync(p.Y, 0, (size_t)mm * ldy * sizeof(float), st));
+            c->pdl_next = false;
+        }
     }
-    return nx;
+    auto kern = e == tc::kEpiStore ? tc2::gemm_tc2_kernel<tc::kEpiStore>
+                : e == tc::kEpiAtomic ? tc2::gemm_tc2_kernel<tc::kEpiAtomic>
+                : e == tc::kEpiSwiglu ? tc2::gemm_tc2_kernel<tc::kEpiSwiglu>
+                                      : tc2::gemm_tc2_kernel<tc::kEpiScatterAtomic>;
+    Launch guard(c, st, kClsGemmTc);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * tiles * p.ksplit);
+    cfg.blockDim = dim3(320);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = (c->use_pdl && !c->profiling && c->pdl_next) ? 2 : 1;
+    c->pdl_next = true;
+    CU_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmBh, tmBl, p));
+    return FIRST_OK;
 }
 
 // Y (+)= X . W^T on the tensor cores.  Xh/Xl: [m][K] bf16 hi/lo activations (compact rows).
 //   epi kEpiStore: Y[j*ldy+f] = ..;  kEpiAtomic: Y zeroed here, then reduced into;
 //   kEpiScatterAtomic: Y[idx[j]*ldy+f] += ..
-// nx: the weights the next projection of the step reads first (prefetched into L2 by this one's idle producer).
 int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmA2, int n_out, int K,
                    const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int epi, float* Y, int64_t ldy,
                    const int32_t* idx, bool pre_zeroed, float* act = nullptr, __nv_bfloat16* act_hi = nullptr,
-                   __nv_bfloat16* act_lo = nullptr, const tc::NextWeights* nx = nullptr) {
+                   __nv_bfloat16* act_lo = nullptr, const int32_t* m_dev = nullptr) {
     int rc;
-    static const tc::NextWeights kNone{};
     for (int r0 = 0; r0 < m; r0 += 256) {
         const int mm = std::min(256, m - r0);
+        if (tc2_wanted(c, mm, n_out, epi)) {  // many rows: a CTA pair per unit shares the activation tiles
+            if ((rc = launch_gemm_tc2(c, st, epi == tc::kEpiSwiglu ? tmA2 : tmA, n_out, K, Xh + (size_t)r0 * K,
+                                      Xl + (size_t)r0 * K, mm, r0, epi,
+                                      Y ? Y + (epi == tc::kEpiScatterAtomic ? 0 : (size_t)r0 * ldy) : nullptr, ldy,
+                                      idx ? idx + r0 : nullptr, pre_zeroed, act ? act + (size_t)r0 * n_out : nullptr,
+                                      act_hi ? act_hi + (size_t)r0 * n_out : nullptr,
+                                      act_lo ? act_lo + (size_t)r0 * n_out : nullptr, m_dev)))
+                return rc;
+            continue;
+        }
         const TcShape t = tc_shape(c, n_out, K, mm, epi);
         tc::GemmParams p{};
         p.n_out = n_out; p.K = K; p.m = mm;
@@ -362,6 +418,8 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.idx = idx ? idx + r0 : nullptr;
         p.flags = c->flags;
         p.stamp = stamp_slot(c, kClsGemmTc);
+        p.m_dev = m_dev;
+        p.row0 = r0;
         CUtensorMap tmBh, tmBl;
         if ((rc = make_map(&tmBh, Xh + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
         if ((rc = make_map(&tmBl, Xl + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
@@ -379,8 +437,7 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
                     : e == tc::kEpiAtomic ? tc::gemm_tc_kernel<tc::kEpiAtomic>
                     : e == tc::kEpiSwiglu ? tc::gemm_tc_kernel<tc::kEpiSwiglu>
                                           : tc::gemm_tc_kernel<tc::kEpiScatterAtomic>;
-        const tc::NextWeights& nxr = (nx && r0 + 256 >= m) ? *nx : kNone;  // the last launch of this projection
-        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(320), smem, tmA, tmA2, tmBh, tmBl, nxr, p))) return rc;
+        if ((rc = launch_k(c, st, kClsGemmTc, kern, dim3(grid), dim3(320), smem, tmA, tmA2, tmBh, tmBl, p))) return rc;
     }
     return FIRST_OK;
 }
@@ -410,20 +467,24 @@ int tc_setup(first_ctx* c) {
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiScatterAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
     CU_TRY(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::kEpiSwiglu>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc2::gemm_tc2_kernel<tc::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTc2SmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc2::gemm_tc2_kernel<tc::kEpiAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTc2SmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc2::gemm_tc2_kernel<tc::kEpiScatterAtomic>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTc2SmemMax));
+    CU_TRY(cudaFuncSetAttribute(tc2::gemm_tc2_kernel<tc::kEpiSwiglu>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTc2SmemMax));
     c->tc_ready = true;
     return FIRST_OK;
 }
 
 template <typename WT, int EPI>
 int launch_gemv(first_ctx* c, cudaStream_t st, const void* W, int n_out, int K, const float* X, int m, float* Y,
-                int64_t ldy, const int32_t* idx) {
+                int64_t ldy, const int32_t* idx, const int32_t* m_dev) {
     const int blocks = std::min((n_out + 7) / 8, c->n_sm * 8);
     for (int r0 = 0; r0 < m; r0 += 8) {
         const int rv = std::min(8, m - r0);
         const WT* w = static_cast<const WT*>(W);
         auto kern = rv == 1 ? gemv_rows<WT, 1, EPI> : rv == 2 ? gemv_rows<WT, 2, EPI>
                     : rv <= 4 ? gemv_rows<WT, 4, EPI> : gemv_rows<WT, 8, EPI>;
-        int rc = launch_k(c, st, kClsGemv, kern, dim3(blocks), dim3(256), 0, w, n_out, K, X, r0, rv, Y, ldy, idx);
+        int rc = launch_k(c, st, kClsGemv, kern, dim3(blocks), dim3(256), 0, w, n_out, K, X, r0, rv, m_dev, Y, ldy, idx);
         if (rc) return rc;
     }
     return FIRST_OK;
@@ -443,12 +504,12 @@ LayerKv layer_kv(const first_kv_cache* kv, int l, int B) {
 
 template <typename KT, int HD>
 int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* kc, const KT* vc,
-                         const LayerKv* kv, const int32_t* len_l, const int32_t* idx) {
+                         const LayerKv* kv, const int32_t* len_l, const int32_t* idx, const int32_t* m_dev) {
     dim3 grid(S, c->d.n_kv_heads, m);
 #define FIRST_ATTN_CASE(G)                                                                                  \
     case G:                                                                                                 \
         return launch_k(c, st, kClsAttn, attn_split_simple<KT, HD, G>, grid, dim3(128), 0, c->q, kc, vc,    \
-                        kv->cap_total, kv->slab_off, len_l, kv->slab_cap, idx, c->d.n_q_heads, c->o_part,   \
+                        kv->cap_total, kv->slab_off, len_l, kv->slab_cap, idx, m_dev, c->d.n_q_heads, c->o_part,   \
                         c->ml_part);
     switch (c->group) {
         FIRST_ATTN_CASE(1)
@@ -464,12 +525,12 @@ int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* 
 
 template <typename KT>
 int launch_attn_simple(first_ctx* c, cudaStream_t st, int S, int m, const void* kc, const void* vc,
-                       const LayerKv* kv, const int32_t* len_l, const int32_t* idx) {
+                       const LayerKv* kv, const int32_t* len_l, const int32_t* idx, const int32_t* m_dev) {
     const KT *k = static_cast<const KT*>(kc), *v = static_cast<const KT*>(vc);
     switch (c->d.head_dim) {
-        case 32: return launch_attn_simple_g<KT, 32>(c, st, S, m, k, v, kv, len_l, idx);
-        case 64: return launch_attn_simple_g<KT, 64>(c, st, S, m, k, v, kv, len_l, idx);
-        case 128: return launch_attn_simple_g<KT, 128>(c, st, S, m, k, v, kv, len_l, idx);
+        case 32: return launch_attn_simple_g<KT, 32>(c, st, S, m, k, v, kv, len_l, idx, m_dev);
+        case 64: return launch_attn_simple_g<KT, 64>(c, st, S, m, k, v, kv, len_l, idx, m_dev);
+        case 128: return launch_attn_simple_g<KT, 128>(c, st, S, m, k, v, kv, len_l, idx, m_dev);
         default: return FIRST_E_UNSUPPORTED;
     }
 }
@@ -491,7 +552,7 @@ template <int HD, int G, bool PAIR = false>
 int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorMap& tk, const CUtensorMap& tv,
                        const LayerKv* kv, const void* kc, const void* vc, int C, float* out,
                        __nv_bfloat16* out_hi, __nv_bfloat16* out_lo, bool fuse_rope, float qscale,
-                       const tc::NextWeights& nx) {
+                       const int32_t* m_dev) {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     attn::RopeFuse rf{};
     if (fuse_rope) {
@@ -502,8 +563,8 @@ int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorM
         rf.v_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(vc));
     }
     return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G, PAIR>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
-                    c->rowinfo, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
-                    out_hi, out_lo, c->flags, rf, nx);
+                    c->rowinfo, m_dev, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
+                    out_hi, out_lo, c->flags, rf);
 }
 
 template <int HD, int G>
@@ -528,10 +589,7 @@ int attn_mma_setup(first_ctx* c) {
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const LayerKv* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
-                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair = false,
-                    const tc::NextWeights* nxp = nullptr) {
-    static const tc::NextWeights kNone{};
-    const tc::NextWeights& nx = nxp ? *nxp : kNone;
+                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair, const int32_t* m_dev) {
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -553,13 +611,13 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     dim3 grid(S, d.n_kv_heads, m);
 #define FIRST_ATTN_PAIR(HD, G)                            \
     if (pair && d.head_dim == HD && c->group == G)        \
-        return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale, nx);
+        return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale, m_dev);
     FIRST_ATTN_PAIR(128, 1) FIRST_ATTN_PAIR(128, 2) FIRST_ATTN_PAIR(128, 3) FIRST_ATTN_PAIR(128, 4)
     FIRST_ATTN_PAIR(64, 1) FIRST_ATTN_PAIR(64, 2) FIRST_ATTN_PAIR(64, 3) FIRST_ATTN_PAIR(64, 4)
 #undef FIRST_ATTN_PAIR
 #define FIRST_ATTN_MMA(HD, G)                 \
     if (d.head_dim == HD && c->group == G)    \
-        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale, nx);
+        return launch_attn_mma_hg<HD, G>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, fuse_rope, qscale, m_dev);
     FIRST_ATTN_MMA(128, 1) FIRST_ATTN_MMA(128, 2) FIRST_ATTN_MMA(128, 3) FIRST_ATTN_MMA(128, 4) FIRST_ATTN_MMA(128, 8)
     FIRST_ATTN_MMA(64, 1) FIRST_ATTN_MMA(64, 2) FIRST_ATTN_MMA(64, 3) FIRST_ATTN_MMA(64, 4) FIRST_ATTN_MMA(64, 8)
 #undef FIRST_ATTN_MMA
@@ -573,15 +631,14 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
 template <typename WT>
 int project(first_ctx* c, cudaStream_t st, bool use_tc, const void* W, const CUtensorMap* tm, int n_out, int K,
             const float* X, const __nv_bfloat16* Xh, const __nv_bfloat16* Xl, int m, int out_mode, float* Y,
-            int64_t ldy, const int32_t* idx, bool allow_split = true, bool pre_zeroed = false,
-            const tc::NextWeights* nx = nullptr) {
+            int64_t ldy, const int32_t* idx, const int32_t* m_dev, bool allow_split = true, bool pre_zeroed = false) {
     if (use_tc) {
         const int epi = out_mode == 1 ? tc::kEpiScatterAtomic : (allow_split ? tc::kEpiAtomic : tc::kEpiStore);
         return launch_gemm_tc(c, st, *tm, *tm, n_out, K, Xh, Xl, m, epi, Y, ldy, idx, pre_zeroed, nullptr, nullptr,
-                              nullptr, nx);
+                              nullptr, m_dev);
     }
-    if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx);
-    return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr);
+    if (out_mode == 1) return launch_gemv<WT, kScatterAdd>(c, st, W, n_out, K, X, m, Y, ldy, idx, m_dev);
+    return launch_gemv<WT, kStore>(c, st, W, n_out, K, X, m, Y, ldy, nullptr, m_dev);
 }
 
 template <typename WT>
@@ -624,10 +681,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                                    cudaMemcpyDeviceToDevice, st));
             c->pdl_next = false;
         }
-        const int m = c->cnt_h[l];
+        const int m = c->cnt_h[l];  // launch rows: the layer's active-row count, or an upper bound of it
         if (m == 0) continue;  // every sequence skips this layer: no launch at all
         const bool t = tc_for(m);
         const int32_t* idx = c->idx + (size_t)l * B;
+        const int32_t* m_dev = c->cnt + l;  // the count itself, read by the kernels
         int32_t* len_l = kv->len + (size_t)l * B;
         const LayerKv lkv = layer_kv(kv, l, B);
         float* f32 = t ? nullptr : c->xn;
@@ -636,28 +694,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         const bool zero_qkv = t;  // (cleared even when a projection ends up with one K range and plain stores)
         const bool fused_ffn = t && c->fuse_swiglu && (F % 64 == 0) && m <= 256;
         const bool zero_gu = t && !fused_ffn;
-        // What each kernel of this layer asks the memory system to fetch for the projection after it (tensor-core
-        // path only): QKV -> all of W_o; attention -> the head of W_gate_up; gate/up -> the head of W_down;
-        // down -> the head of the next active layer's W_qkv (or of lm_head).
-        tc::NextWeights nx_o{}, nx_gu{}, nx_down{}, nx_after{};
-        if (t && (c->pf_depth > 0 || c->pf_attn_depth > 0 || c->pf_o) && !ph) {
-            nx_o = next_weights(c, &c->tm_wo[l], nullptr, D, c->qd, m, tc::kEpiScatterAtomic, c->pf_o ? (1 << 20) : 0);
-            if (fused_ffn)
-                nx_gu = next_weights(c, &c->tm_wgu[l], &c->tm_wgu64[l], F, D, m, tc::kEpiSwiglu, c->pf_attn_depth);
-            else
-                nx_gu = next_weights(c, &c->tm_wgu[l], nullptr, 2 * F, D, m, tc::kEpiAtomic, c->pf_attn_depth);
-            nx_down = next_weights(c, &c->tm_wd[l], nullptr, D, F, m, tc::kEpiScatterAtomic, c->pf_depth);
-            int ln = l + 1;
-            while (ln < L && c->cnt_h[ln] == 0) ++ln;
-            if (ln < L) {
-                if (tc_for(c->cnt_h[ln]))
-                    nx_after = next_weights(c, &c->tm_wqkv[ln], nullptr, c->qkvd, D, c->cnt_h[ln], tc::kEpiAtomic, c->pf_depth);
-            } else if (tc_for(B) && (logits || next_tokens)) {
-                nx_after = next_weights(c, &c->tm_lm, nullptr, V, D, B, tc::kEpiStore, c->pf_depth);
-            }
-        }
         // ---- attention half
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->attn_norm[l],
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, m_dev, D, c->attn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_qkv ? c->qkv : nullptr, c->qkvd, static_cast<int32_t*>(nullptr),
                            fuse_rope ? lkv.slab_cap : nullptr, fuse_rope ? c->rowinfo : nullptr,
                            fuse_rope ? static_cast<const int32_t*>(len_l) : nullptr, fuse_rope ? lkv.slab_off : nullptr,
@@ -668,50 +706,50 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                            route_here ? ph->tokscore + (size_t)l * ph->stride + ph->g0 : nullptr)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
-                              c->qkv, c->qkvd, nullptr, true, zero_qkv, &nx_o)))
+                              c->qkv, c->qkvd, nullptr, m_dev, true, zero_qkv)))
             return rc;
         // The tuned attention kernel rotates q itself and appends the new token's key and value (its
         // row facts come from the norm kernel above); the general path has a kernel for that.
         if (!fuse_rope &&
             (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3((d.n_q_heads + 2 * d.n_kv_heads + 7) / 8, m), dim3(hd / 2, 8),
-                           0, c->qkv, idx, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
+                           0, c->qkv, idx, m_dev, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
                            lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0)))
             return rc;
         if (mma_attn) {
             if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], &lkv, len_l, idx, t ? nullptr : c->att, xh, xl,
-                                      fuse_rope, qscale, pair_rows, &nx_gu)))
+                                      fuse_rope, qscale, pair_rows, m_dev)))
                 return rc;
         } else {
-            if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], &lkv, len_l, idx))) return rc;
+            if ((rc = launch_attn_simple<WT>(c, st, S, m, kv->k[l], kv->v[l], &lkv, len_l, idx, m_dev))) return rc;
             if ((rc = launch_k(c, st, kClsAttnCombine, attn_combine, dim3(m * d.n_q_heads), dim3(128), 0, c->o_part,
-                               c->ml_part, S, hd, t ? nullptr : c->att, xh, xl)))
+                               c->ml_part, m_dev, d.n_q_heads, S, hd, t ? nullptr : c->att, xh, xl)))
                 return rc;
         }
         if ((rc = project<WT>(c, st, t, c->wo[l], t ? &c->tm_wo[l] : nullptr, D, c->qd, c->att, c->xh, c->xl, m, 1, c->x,
-                              D, idx)))
+                              D, idx, m_dev)))
             return rc;
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, D, c->ffn_norm[l],
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, m_dev, D, c->ffn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, lkv.slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
                            static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
             if ((rc = launch_gemm_tc(c, st, c->tm_wgu64[l], c->tm_wgu[l], F, D, c->xh, c->xl, m, tc::kEpiSwiglu, nullptr, 0, nullptr,
-                                     false, nullptr, c->acth, c->actl, &nx_down)))
+                                     false, nullptr, c->acth, c->actl, m_dev)))
                 return rc;
         } else {
             if ((rc = project<WT>(c, st, t, c->w_gate_up[l], t ? &c->tm_wgu[l] : nullptr, 2 * F, D, c->xn, c->xh, c->xl,
-                                  m, 0, c->gu, 2 * F, nullptr, true, zero_gu, &nx_down)))
+                                  m, 0, c->gu, 2 * F, nullptr, m_dev, true, zero_gu)))
                 return rc;
             if ((rc = launch_k(c, st, kClsSiluMul, silu_mul, dim3(std::min((m * F + 255) / 256, c->n_sm * 8)),
-                               dim3(256), 0, c->gu, m, F, t ? nullptr : c->act, t ? c->acth : nullptr,
+                               dim3(256), 0, c->gu, m, m_dev, F, t ? nullptr : c->act, t ? c->acth : nullptr,
                                t ? c->actl : nullptr)))
                 return rc;
         }
         if ((rc = project<WT>(c, st, t, c->w_down[l], t ? &c->tm_wd[l] : nullptr, D, F, c->act, c->acth, c->actl, m, 1,
-                              c->x, D, idx, true, false, &nx_after)))
+                              c->x, D, idx, m_dev)))
             return rc;
     }
     if (ph) return FIRST_OK;  // a prefill chunk ends here: logits are taken once, from the last prompt tokens
@@ -731,13 +769,13 @@ int logits_tail(first_ctx* c, cudaStream_t st, int B, float* logits, int32_t* ne
     float* lg = logits ? logits : (next_tokens ? c->logits_int : nullptr);
     if (lg) {
         const bool t = tc_for(B);
-        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, D, c->final_norm,
+        if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, nullptr, D, c->final_norm,
                            d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
                            nullptr, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
                            static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
             return rc;
         if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
-                              nullptr, false)))
+                              nullptr, nullptr, false)))
             return rc;
     }
     if (next_tokens && lg && c->sample_k > 1)
@@ -819,7 +857,8 @@ int first_create(const first_model_desc* desc, const first_weights* w, first_ctx
         (rc = dev_alloc(&c->cs, MB * (d.head_dim / 2))) || (rc = dev_alloc(&c->inv_freq, (size_t)d.head_dim / 2)) ||
         (rc = dev_alloc(&c->idx, MB * d.n_layers)) || (rc = dev_alloc(&c->cnt, (size_t)d.n_layers)) ||
         (rc = dev_alloc(&c->slot, MB * d.n_layers)) || (rc = dev_alloc(&c->flags, (size_t)1)) ||
-        (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)) || (rc = dev_alloc(&c->rowinfo, MB)))
+        (rc = dev_alloc(&c->ticket, MB * d.n_kv_heads)) || (rc = dev_alloc(&c->rowinfo, MB)) ||
+        (rc = dev_alloc(&c->mask_dev, MB * d.n_layers)))
         return fail(rc);
     if (cudaMemset(c->ticket, 0, MB * d.n_kv_heads * sizeof(uint32_t)) != cudaSuccess) return fail(FIRST_E_CUDA);
     if ((rc = dev_alloc(&c->pf_cu, MB + 1)) || (rc = dev_alloc(&c->pf_tok, MB)) || (rc = dev_alloc(&c->pf_cap, MB)) ||
@@ -851,7 +890,7 @@ int first_destroy(first_ctx* c) {
     void* ptrs[] = {c->x, c->xn, c->qkv, c->q, c->att, c->gu, c->act, c->o_part, c->logits_int, c->tokscore,
                     c->ml_part, c->cs, c->inv_freq, c->idx, c->cnt, c->slot, c->flags, c->xh, c->xl, c->acth, c->actl, c->ticket, c->rowinfo,
                     c->pf_cu, c->pf_tok, c->pf_cap, c->pf_pos, c->pf_len, c->pf_off, c->pf_ones, c->x_last, c->pf_score,
-                    c->stamps};
+                    c->stamps, c->mask_dev};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -895,9 +934,6 @@ int first_set_mask(first_ctx* c, const uint8_t* mask, int32_t B, void* stream) {
     if (B > c->d.max_batch) return FIRST_E_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     c->has_mask = false;
-    c->plan_version += 1;  // step graphs recorded under the previous plan must not be replayed
-    for (auto& e : c->graphs) cudaGraphExecDestroy(e.exec);
-    c->graphs.clear();
     FIRST_LAUNCH(kClsPlan, (plan_compact<<<c->d.n_layers, 32, 0, st>>>(mask, B, c->d.n_layers, c->idx, c->cnt, c->slot, c->flags)));
     int rc = check_launch(c);
     if (rc) return rc;
@@ -906,6 +942,36 @@ int first_set_mask(first_ctx* c, const uint8_t* mask, int32_t B, void* stream) {
     CU_TRY(cudaMemcpyAsync(&fl, c->flags, sizeof fl, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
     if (fl & FIRST_FLAG_BAD_MASK) return FIRST_E_DEVICE_FLAG;
+    c->B = B;
+    c->has_mask = true;  // launch rows = the exact counts; recorded step graphs are looked up by them
+    return FIRST_OK;
+}
+
+int first_set_mask_host(first_ctx* c, const uint8_t* mask, int32_t B, void* stream) {
+    if (!c || !mask || B <= 0) return FIRST_E_ARG;
+    if (B > c->d.max_batch) return FIRST_E_CAPACITY;
+    const int L = c->d.n_layers;
+    std::vector<int32_t> cnt(L, 0);
+    for (int b = 0; b < B; ++b)
+        for (int l = 0; l < L; ++l) {
+            const uint8_t mk = mask[(size_t)b * L + l];
+            if (mk > 1) return FIRST_E_ARG;
+            cnt[l] += mk;
+        }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_TRY(cudaStreamIsCapturing(st, &cap));
+    if (cap != cudaStreamCaptureStatusNone) return FIRST_E_STATE;
+    c->has_mask = false;
+    // pageable source: the runtime takes its own copy before returning, and does not wait for the stream
+    CU_TRY(cudaMemcpyAsync(c->mask_dev, mask, (size_t)B * L, cudaMemcpyHostToDevice, st));
+    FIRST_LAUNCH(kClsPlan, (plan_compact<<<L, 32, 0, st>>>(c->mask_dev, B, L, c->idx, c->cnt, c->slot, c->flags)));
+    int rc = check_launch(c);
+    if (rc) return rc;
+    // Launch rows: the count rounded up to the next multiple of 16 (the projections pad to that anyway).  The
+    // kernels read the exact count from device memory, so a batch change that keeps every layer inside its
+    // bucket finds its recorded step graph again.
+    for (int l = 0; l < L; ++l) c->cnt_h[l] = cnt[l] == 0 ? 0 : std::min<int>(B, (cnt[l] + 15) / 16 * 16);
     c->B = B;
     c->has_mask = true;
     return FIRST_OK;
@@ -956,13 +1022,16 @@ int first_decode_step(first_ctx* c, const int32_t* tokens, const first_kv_cache*
     if (kv->per_layer)
         for (int l = 0; l < c->d.n_layers; ++l)
             key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(kv->cap_total_l[l])));
-    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->plan_version)));
+    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->plan_version)));  // options, sampling
+    key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->B)));
+    for (int l = 0; l < c->d.n_layers; ++l)  // the launch sequence is a function of the rows launched per layer
+        key.push_back(reinterpret_cast<const void*>(static_cast<uintptr_t>(c->cnt_h[l])));
     for (int l = 0; l < c->d.n_layers; ++l) { key.push_back(kv->k[l]); key.push_back(kv->v[l]); }
     first_ctx::StepGraph* g = nullptr;
     for (auto& e : c->graphs)
         if (e.key == key) { g = &e; break; }
     if (!g) {
-        if (c->graphs.size() >= 8) {  // drop the least recently used
+        if (c->graphs.size() >= 16) {  // drop the least recently used
             size_t lru = 0;
             for (size_t i = 1; i < c->graphs.size(); ++i)
                 if (c->graphs[i].last_use < c->graphs[lru].last_use) lru = i;
@@ -1125,6 +1194,14 @@ int first_selftest_wait_expiry(first_ctx* c, int32_t polls, int32_t* returned, i
 
 int64_t first_launch_count(const first_ctx* c) { return c ? c->launches : 0; }
 
+int first_get_desc(const first_ctx* c, first_model_desc* out) {
+    if (!c || !out) return FIRST_E_ARG;
+    *out = c->d;
+    return FIRST_OK;
+}
+
+int64_t first_graph_count(const first_ctx* c) { return c ? (int64_t)c->graphs.size() : 0; }
+
 int first_profile(first_ctx* c, int32_t enable) {
     if (!c) return FIRST_E_ARG;
     c->profiling = enable != 0;
@@ -1209,9 +1286,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
-    else if (!std::strcmp(name, "pf_depth")) c->pf_depth = value >= 0 ? (int)value : 0;
-    else if (!std::strcmp(name, "pf_attn_depth")) c->pf_attn_depth = value >= 0 ? (int)value : 0;
-    else if (!std::strcmp(name, "pf_o")) c->pf_o = value > 0;
+    else if (!std::strcmp(name, "tc2_min_rows")) c->tc2_min_rows = value > 0 ? (int)value : 0;
     else if (!std::strcmp(name, "stamp")) {
         c->stamp_on = value > 0;
         if (c->stamp_on && !c->stamps) {

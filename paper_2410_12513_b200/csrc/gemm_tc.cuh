@@ -51,42 +51,9 @@ struct GemmParams {
     __nv_bfloat16* act_hi;   // [m][n_out] bfloat16 hi/lo split or NULL
     __nv_bfloat16* act_lo;
     uint64_t* stamp;         // in-step timing slot or NULL
+    const int32_t* m_dev;    // active-row count in device memory (m is a host-side upper bound of it) or NULL
+    int row0;                // first compact row of this launch (launches take 256 rows each)
 };
-
-// What the NEXT weight-streaming kernel of the step will read first.  A kernel that has finished asking for
-// its own tiles (and so leaves HBM idle during its epilogue, the kernel boundary and the next kernel's
-// start-up) asks the memory system to bring the first `depth` k-blocks of every work unit of the next
-// projection into L2; that projection then starts on L2 hits.  The work units are enumerated exactly as
-// gemm_tc_kernel enumerates them.  mode 0: nothing; 1: tiles of mt x 128 rows; 2: gate|up pairs (two boxes
-// of `rows` rows, the second n_out rows further down).  A prefetch has no architectural effect: a wrong
-// guess costs bandwidth, never correctness.
-struct NextWeights {
-    CUtensorMap map;
-    int mode, tiles, ksplit, kblocks, depth, rows, n_out, mt;
-};
-
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
-}
-
-// Called by ONE thread of CTA `cta` of `n_cta`: that CTA's share of the next projection's work units.
-__device__ __forceinline__ void prefetch_next_weights(const NextWeights& nx, int cta, int n_cta) {
-    if (nx.mode == 0) return;
-    const int units = nx.tiles * nx.ksplit;
-    for (int u = cta; u < units; u += n_cta) {
-        const int tile = u / nx.ksplit, split = u - tile * nx.ksplit;
-        const int kb0 = (int)((int64_t)nx.kblocks * split / nx.ksplit);
-        const int kb1 = min((int)((int64_t)nx.kblocks * (split + 1) / nx.ksplit), kb0 + nx.depth);
-        for (int kb = kb0; kb < kb1; ++kb) {
-            if (nx.mode == 2) {
-                tma_prefetch_2d(&nx.map, kb * kBlockK, tile * nx.rows);
-                tma_prefetch_2d(&nx.map, kb * kBlockK, nx.n_out + tile * nx.rows);
-            } else {
-                for (int a = 0; a < nx.mt; ++a) tma_prefetch_2d(&nx.map, kb * kBlockK, (tile * nx.mt + a) * kBlockM);
-            }
-        }
-    }
-}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -167,8 +134,7 @@ template <int EPI>
 __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                       const __grid_constant__ CUtensorMap tmA2,
                                                       const __grid_constant__ CUtensorMap tmBh,
-                                                      const __grid_constant__ CUtensorMap tmBl,
-                                                      const __grid_constant__ NextWeights nx, const GemmParams p) {
+                                                      const __grid_constant__ CUtensorMap tmBl, const GemmParams p) {
     const Stamp stamp_guard(p.stamp);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -254,8 +220,6 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
                 tma_load_2d(sa + a_bytes, &tmBh, full_bar(s), kc, 0);
                 if (p.use_lo) tma_load_2d(sa + a_bytes + b_bytes, &tmBl, full_bar(s), kc, 0);
             }
-            // every weight tile of this CTA has been asked for: from here on it leaves HBM idle
-            if (!abort_s) prefetch_next_weights(nx, (int)blockIdx.x, (int)gridDim.x);
             // This lane does not reach the CTA's final barrier before every copy it issued has landed (the last
             // use of each stage; earlier uses were consumed before their stage was refilled).  It does so
             // whether or not any role has given up and whichever role notices first: the CTA's shared memory
@@ -302,6 +266,8 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         pdl_wait();  // the epilogue reduces into buffers the previous kernels own
+        // rows that exist: the columns beyond them were computed from stale activation rows and are dropped
+        const int m_act = p.m_dev ? max(0, min(p.m, __ldg(p.m_dev) - p.row0)) : p.m;
         const bool ok = mbar_wait(tmem_full_bar, 0u, &abort_s, p.flags) && !abort_s;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const bool run = ok && nkb > 0;
@@ -318,7 +284,7 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             const int j = c0 + c;
-                            if (j < p.m) {
+                            if (j < m_act) {
                                 const float g = __uint_as_float(vg[c]);
                                 const float y = g / (1.f + expf(-g)) * __uint_as_float(vu[c]);
                                 const size_t o = (size_t)j * p.n_out + f;
@@ -359,7 +325,7 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
                         const int j = c0 + c;
-                        if (j < p.m) {
+                        if (j < m_act) {
                             const float g = __uint_as_float(v[c]);
                             const float y = g / (1.f + expf(-g)) * ub[c * 64 + gl];
                             const size_t o = (size_t)j * p.n_out + f;
@@ -384,7 +350,7 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             const int j = c0 + c;
-                            if (j < p.m) {
+                            if (j < m_act) {
                                 const float val = __uint_as_float(v[c]);
                                 if (EPI == kEpiStore) p.Y[(size_t)j * p.ldy + f] = val;
                                 else if (EPI == kEpiAtomic) atomicAdd(p.Y + (size_t)j * p.ldy + f, val);

@@ -16,11 +16,15 @@ enum GemvEpilogue { kStore = 0, kScatterAdd = 1 };
 template <typename WT, int R, int EPI>
 __global__ void __launch_bounds__(256) gemv_rows(const WT* __restrict__ W, int n_out, int K,
                                                  const float* X, int r0, int rows_valid,
+                                                 const int32_t* __restrict__ m_dev,
                                                  float* __restrict__ Y, int64_t ldy, const int32_t* __restrict__ idx,
                                                  uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
+    // m_dev: the active-row count in device memory (the host launches for an upper bound of it)
+    if (m_dev) rows_valid = min(rows_valid, __ldg(m_dev) - r0);
     pdl_wait();
+    if (rows_valid <= 0) return;
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;

@@ -65,7 +65,11 @@ __device__ __forceinline__ void split_store4(const float (&y)[4], __nv_bfloat16*
 //   router:   (prompt processing) the row is also what the layer's router reads: its score
 //             z = router_w . x[b] (+ bias) goes to tok_out[i], as sigmoid(z) in the paper's order
 //             (mean of per-token sigmoids) or as z in the pooled order, like router_token_scores.
-__global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32_t* __restrict__ idx, int D,
+// m_dev (all the per-layer kernels have it): the layer's active-row count in device memory.  The grid is sized
+// from a host-side upper bound of it (so that a recorded launch sequence survives small changes of the batch);
+// work items beyond the count leave at once.  NULL = every row of the grid is live.
+__global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32_t* __restrict__ idx,
+                                                     const int32_t* __restrict__ m_dev, int D,
                                                      const float* __restrict__ gain, float eps, float* __restrict__ out,
                                                      __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                      float* __restrict__ zero_row, int zero_cols,
@@ -83,6 +87,10 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
     constexpr int kMaxV = 4;
     pdl_trigger();
     const int i = blockIdx.x, nt = blockDim.x;
+    if (m_dev && i >= __ldg(m_dev)) {  // (the plan is fixed between first_set_mask calls)
+        pdl_wait();  // a grid must not complete before its predecessor has: later kernels rely on that chain
+        return;
+    }
     float4 g[kMaxV];
     const int nv = D / 4;
 #pragma unroll
@@ -170,6 +178,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
 // A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
 __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32_t* __restrict__ idx,
+                                                  const int32_t* __restrict__ m_dev,
                                                   int Hq, int Hkv, int hd, const float2* cs,
                                                   float qscale, float* __restrict__ q_out, KT* __restrict__ kc,
                                                   KT* __restrict__ vc, int64_t cap_total,
@@ -179,7 +188,9 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                                                   longlong2* __restrict__ rowinfo, int pair, uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
+    const int m = m_dev ? min((int)gridDim.y, __ldg(m_dev)) : (int)gridDim.y;
     pdl_wait();
+    if ((int)blockIdx.y >= m) return;
     const int i = blockIdx.y, head = blockIdx.x * blockDim.y + threadIdx.y, d = threadIdx.x, b = idx[i];
     if (head >= Hq + 2 * Hkv) return;
     if (rowinfo && head == 0 && d == 0) {  // what attention needs to know about this row, in one 16-byte word
@@ -187,7 +198,6 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
         if (pair) {
             // Prompt processing: rows i0, i0+1 that are consecutive tokens of one slab (the first at an even
             // position, both with room) share attention work items: bit 61 marks the first, bit 60 the second.
-            const int m = gridDim.y;
             auto is_pair = [&](int i0) {
                 if (i0 < 0 || i0 + 1 >= m) return false;
                 const int b0 = idx[i0], b1 = idx[i0 + 1];
@@ -230,11 +240,13 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
 }
 
 // act[i][f] = silu(gate) * up from gu[i] = [gate(F) | up(F)]; optional bf16 hi/lo split.
-__global__ void __launch_bounds__(256) silu_mul(const float* gu, int m, int F, float* __restrict__ act,
+__global__ void __launch_bounds__(256) silu_mul(const float* gu, int m, const int32_t* __restrict__ m_dev, int F,
+                                                float* __restrict__ act,
                                                 __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                 uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
+    if (m_dev) m = min(m, __ldg(m_dev));
     pdl_wait();
     const size_t n = (size_t)m * F;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
