@@ -267,6 +267,60 @@ def prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks,
             "note": "prompt tokens as rows of the decode-step kernels, 256 per chunk; weights streamed once per chunk"}
 
 
+def join_leg(torch, job, mask, lens, room, changes=8):
+    """Cost of a batch change between steps: the job's batch decodes through a slab pool laid over the same cache
+    tensors (slabs only for kept (sequence, layer) pairs); then, `changes` times, one sequence leaves, another
+    (same prompt length, another mask row) joins, the plan is rebuilt from the host masks, and the next step runs.
+    Host time of leave + join + commit, and the device time of the first step after the change against a steady
+    step (a change that moves a layer's row count into another bucket of 16 records a new step graph)."""
+    from paper_2410_12513_b200 import FirstPool
+    ctx, B, L = job.ctx, job.B, job.L
+    pool = FirstPool(ctx, B, job.kk, job.vv)
+    caps = [int(n) + room + 1 for n in lens]
+    slots = [pool.join(mask[b], caps[b], None, 0, int(lens[b])) for b in range(B)]
+    pool.commit()
+    stream = job.stream
+
+    def step_ms(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        a, b = job.tok_a, job.tok_b
+        for _ in range(n):
+            ctx.decode_step(a, pool.kv, None, b)
+            a, b = b, a
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    job.tok_a.copy_(job.tok0)
+    step_ms(3)
+    steady = step_ms(8)
+    held0 = pool.stats()[0].sum()
+    rng = np.random.default_rng(11)
+    host_us, first_ms = [], []
+    g0 = ctx.graph_count()
+    for i in range(changes):
+        b = int(rng.integers(0, B))
+        row = mask[int(rng.integers(0, B))]
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        pool.leave(slots[b])
+        slots[b] = pool.join(row, caps[b], None, 0, int(lens[b]))
+        pool.commit()
+        host_us.append((time.perf_counter() - t0) * 1e6)
+        first_ms.append(step_ms(1))
+        step_ms(2)
+    flags = ctx.device_flags()
+    rec = {"steady_ms_per_step_through_pool": steady, "host_us_leave_join_commit_median": float(np.median(host_us)),
+           "first_step_after_change_ms_median": float(np.median(first_ms)),
+           "first_step_after_change_ms_max": float(np.max(first_ms)), "changes": changes,
+           "step_graphs_recorded_during_changes": int(ctx.graph_count() - g0),
+           "kv_rows_held": int(held0), "kv_rows_if_every_layer_had_a_slab": int(sum(caps)) * L, "device_flags": int(flags),
+           "note": "no call of a change waits for the stream; rows held = sum over kept (sequence, layer) slabs"}
+    pool.close()
+    return rec
+
+
 # ----------------------------------------------------------------------------- replicas (N > 1)
 def init_replica():
     """(rank, world, local device index, dist module or None, device for the max-over-ranks tensor).
@@ -683,6 +737,8 @@ def run_cuda(args, wl, shape, mask, lens):
            "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
            "kernel_ms_in_step": in_step, "traced_step_ms": traced_step_ms,
            "kernel_ms_per_step_event_pairs": cls_ms, "route": route}
+    if not args.no_join and rank == 0:
+        out["batch_change"] = join_leg(torch, job, mask, lens, W + K)
     if not args.no_prefill and rank == 0:
         out["prefill"] = prefill_leg(torch, FirstContext, shape, weights, kv, lens, caps, dev, peaks, opts=args.opt)
     job.close()
@@ -723,6 +779,7 @@ def main():
                     help="reduced layer count: a small case for profiler captures, never a benchmark value")
     ap.add_argument("--sweep", action="store_true",
                     help="time six skip fractions 0..50 %% (aligned and independent masks) on this workload instead of three")
+    ap.add_argument("--no-join", action="store_true", help="skip the batch-change leg (slab pool: leave + join + plan rebuild)")
     ap.add_argument("--no-sub", action="store_true", help="skip the sub-records of the other benchmark workloads")
     ap.add_argument("--quick", action="store_true",
                     help="only the main timed loop (for profiler captures): no dense/e2e/per-kernel legs")

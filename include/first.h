@@ -292,7 +292,8 @@ int first_decode_step(first_ctx *ctx, const int32_t *tokens, const first_kv_cach
  *                     (<= max_tokens_per_seq).  src != NULL: the keys/values of the sequence's first
  *                     n_tokens tokens are copied, for the kept layers, from sequence src_seq of cache `src`
  *                     (per_layer = 0, e.g. the cache a first_prefill call filled), len = pos = n_tokens;
- *                     src == NULL: empty slabs, n_tokens must be 0.  *slot = the batch row: the caller
+ *                     src == NULL: nothing is copied; the first n_tokens rows of the new slabs count as
+ *                     present, whatever they hold (0 for empty slabs).  *slot = the batch row: the caller
  *                     feeds the sequence's tokens at tokens[slot] and reads its logits at row slot.
  *                     FIRST_E_CAPACITY: no free batch row, or some kept layer has no free range of
  *                     `capacity` rows (nothing is taken then).
@@ -402,6 +403,9 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *   "tc_mt2_min_rows" from this many active rows on a projection CTA takes two weight tiles per
  *                    activation tile (default: when the activation tiles are so wide that only one
  *                    single-tile CTA would fit per SM, i.e. from 96 rows)
+ *   "tc2_min_rows"   from this many active rows on a tensor-core projection launch runs as CTA pairs (two SMs per
+ *                    unit, cta_group::2 MMA, each SM holding half of the activation rows); default 96, 0 = never
+ *   "tc2_mt2_all"    1 = the CTA-pair kernel takes two weight tiles per unit for the reducing epilogues too
  *   "tc_ksplit_cap"  0 = do not bound the number of K ranges by the reduction traffic
  *   "tc_smem_kb"     shared-memory budget per projection CTA when two CTAs per SM are wanted (110)
  *   "fuse_rope"      0 = a separate kernel rotates q/k and appends the new key/value before attention.

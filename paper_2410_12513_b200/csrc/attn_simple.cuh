@@ -19,7 +19,7 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
                                                          const int32_t* __restrict__ idx,
                                                          const int32_t* __restrict__ m_dev, int Hq,
                                                          float* __restrict__ o_part, float2* __restrict__ ml_part,
-                                                         uint64_t* stamp) {
+                                                         int cap_max, uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
     pdl_wait();
@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(128) attn_split_simple(const float* q, const K
     constexpr int EPL = HD / 32;
     const int S = gridDim.x, s = blockIdx.x, h = blockIdx.y, i = blockIdx.z;
     const int b = idx[i];
-    const int T = min(len_l[b] + 1, slab_cap[b]);  // the new token sits at row len (len itself advances later)
+    const int T = min(len_l[b] + 1, min(slab_cap[b], cap_max));  // the new token sits at row len (len itself advances later)
     const int C = (T + S - 1) / S;
     const int t0 = s * C, t1 = min(T, t0 + C);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

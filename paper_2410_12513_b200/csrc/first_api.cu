@@ -97,7 +97,8 @@ struct first_ctx {
     int stamp_n = 0;
     std::vector<int> stamp_cls;
     // options
-    int tc2_min_rows = 0;   // from this many rows on a projection launch uses the CTA-pair kernel (0 = never)
+    int tc2_min_rows = 96;  // from this many rows on a projection launch uses the CTA-pair kernel (0 = never)
+    int tc2_mt2_all = 0;    // CTA-pair kernel: two weight tiles per unit for the reducing epilogues too
     int max_gemv_rows = -1;
     int attn_simple = -1;
     int tc_use_lo = 1;
@@ -307,7 +308,7 @@ TcShape tc_shape(const first_ctx* c, int n_out, int K, int mm, int epi) {
 
 // The CTA-pair kernel (gemm_tc2.cuh) for launches of many rows.  Units = (group of two 256-row weight tiles, K
 // range); the K ranges fill the SM pairs in whole waves.
-constexpr int kTc2SmemMax = 226 * 1024;
+constexpr int kTc2SmemMax = 231000;  // dynamic bytes; the kernels' static shared memory (about 1 KB) comes on top
 
 bool tc2_wanted(const first_ctx* c, int mm, int n_out, int epi) {
     if (c->tc2_min_rows <= 0 || mm < c->tc2_min_rows || mm > 256) return false;
@@ -324,12 +325,21 @@ int launch_gemm_tc2(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, int n
     p.n_pad = (mm + 31) / 32 * 32;  // half of the activation rows in each CTA, in whole 16-row groups
     p.kblocks = (K + tc::kBlockK - 1) / tc::kBlockK;
     p.use_lo = (c->tc_use_lo && mm <= c->tc_lo_max_rows) ? 1 : 0;
-    p.mt = 2;
+    // Two 256-row weight tiles per unit share every activation tile where the epilogue is cheap (plain stores,
+    // SwiGLU).  The reducing epilogues take one tile per unit: the same SM pairs are then filled with half as many
+    // K ranges, and every K range costs m x n_out float32 reductions (7 M per launch at 192 rows with the larger
+    // units, which alone took 8 us).
+    p.mt = (epi == tc::kEpiStore || epi == tc::kEpiSwiglu || c->tc2_mt2_all) ? 2 : 1;
     p.pair_rows = 0;
-    const int tiles = epi == tc::kEpiSwiglu ? (n_out + 255) / 256 : (n_out + 511) / 512;
+    const int tiles = epi == tc::kEpiSwiglu ? (n_out + 255) / 256 : (n_out + 256 * p.mt - 1) / (256 * p.mt);
     const int stage_bytes = tc::kABytes * p.mt + (p.n_pad / 2) * 128 * (p.use_lo ? 2 : 1);
-    p.stages = std::max(2, std::min(8, (kTc2SmemMax - 2048) / stage_bytes));
-    p.ksplit = tc_ksplit(c, tiles, K, epi, mm, std::max(1, c->n_sm / 2));
+    p.stages = std::max(2, std::min(8, (kTc2SmemMax - 1280) / stage_bytes));
+    // K ranges: as many as keep all units in ONE wave of the SM pairs (one CTA fits per SM here, so a second wave
+    // would pay set-up and epilogue again, back to back), at least four k-blocks each.
+    const int slots = std::max(1, c->n_sm / 2);
+    p.ksplit = 1;
+    if (epi == tc::kEpiAtomic || epi == tc::kEpiScatterAtomic)
+        p.ksplit = std::max(1, std::min(p.kblocks / 4, slots / std::max(tiles, 1)));
     int cols = 32;
     while (cols < p.n_pad) cols *= 2;
     p.acc_cols = cols;
@@ -510,7 +520,7 @@ int launch_attn_simple_g(first_ctx* c, cudaStream_t st, int S, int m, const KT* 
     case G:                                                                                                 \
         return launch_k(c, st, kClsAttn, attn_split_simple<KT, HD, G>, grid, dim3(128), 0, c->q, kc, vc,    \
                         kv->cap_total, kv->slab_off, len_l, kv->slab_cap, idx, m_dev, c->d.n_q_heads, c->o_part,   \
-                        c->ml_part);
+                        c->ml_part, c->d.max_tokens_per_seq);
     switch (c->group) {
         FIRST_ATTN_CASE(1)
         FIRST_ATTN_CASE(2)
@@ -703,7 +713,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
                            // prompt chunks (all rows active, idx[i] = i): router l scores the rows it normalises
                            route_here ? ph->router_w + (size_t)l * D : nullptr,
                            route_here && ph->router_b ? ph->router_b + l : nullptr, route_here ? ph->mode : 0,
-                           route_here ? ph->tokscore + (size_t)l * ph->stride + ph->g0 : nullptr)))
+                           route_here ? ph->tokscore + (size_t)l * ph->stride + ph->g0 : nullptr, d.max_tokens_per_seq)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->wqkv[l], t ? &c->tm_wqkv[l] : nullptr, c->qkvd, D, c->xn, c->xh, c->xl, m, 0,
                               c->qkv, c->qkvd, nullptr, m_dev, true, zero_qkv)))
@@ -714,7 +724,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3((d.n_q_heads + 2 * d.n_kv_heads + 7) / 8, m), dim3(hd / 2, 8),
                            0, c->qkv, idx, m_dev, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
-                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0)))
+                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0,
+                           d.max_tokens_per_seq)))
             return rc;
         if (mma_attn) {
             if ((rc = launch_attn_mma(c, st, m, kv->k[l], kv->v[l], &lkv, len_l, idx, t ? nullptr : c->att, xh, xl,
@@ -732,7 +743,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
         // ---- feed-forward half (its norm kernel also advances the cache length of the rows it handles)
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(m), dim3(norm_threads), 0, c->x, idx, m_dev, D, c->ffn_norm[l],
                            d.rms_eps, f32, xh, xl, zero_gu ? c->gu : nullptr, 2 * F, len_l, lkv.slab_cap, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
-                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
+                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr), d.max_tokens_per_seq)))
             return rc;
         if (fused_ffn) {
             // gate/up projection with silu(gate)*up applied in its epilogue: the activation is written once
@@ -772,7 +783,7 @@ int logits_tail(first_ctx* c, cudaStream_t st, int B, float* logits, int32_t* ne
         if ((rc = launch_k(c, st, kClsRmsnorm, rmsnorm_rows, dim3(B), dim3(norm_threads), 0, c->x, nullptr, nullptr, D, c->final_norm,
                            d.rms_eps, t ? nullptr : c->xn, t ? c->xh : nullptr, t ? c->xl : nullptr, nullptr, 0, nullptr,
                            nullptr, static_cast<longlong2*>(nullptr), static_cast<const int32_t*>(nullptr), static_cast<const int64_t*>(nullptr), static_cast<uint32_t*>(nullptr),
-                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr))))
+                           static_cast<const float*>(nullptr), static_cast<const float*>(nullptr), 0, static_cast<float*>(nullptr), d.max_tokens_per_seq)))
             return rc;
         if ((rc = project<WT>(c, st, t, c->lm_head, t ? &c->tm_lm : nullptr, V, D, c->xn, c->xh, c->xl, B, 0, lg, V,
                               nullptr, nullptr, false)))
@@ -1286,7 +1297,8 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;
     else if (!std::strcmp(name, "tc_ksplit_cap")) c->tc_ksplit_cap = value != 0;
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
-    else if (!std::strcmp(name, "tc2_min_rows")) c->tc2_min_rows = value > 0 ? (int)value : 0;
+    else if (!std::strcmp(name, "tc2_min_rows")) c->tc2_min_rows = value < 0 ? 96 : (int)value;
+    else if (!std::strcmp(name, "tc2_mt2_all")) c->tc2_mt2_all = value > 0;
     else if (!std::strcmp(name, "stamp")) {
         c->stamp_on = value > 0;
         if (c->stamp_on && !c->stamps) {

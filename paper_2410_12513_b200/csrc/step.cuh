@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
                                                      uint32_t* __restrict__ flags,
                                                      const float* __restrict__ router_w,
                                                      const float* __restrict__ router_b, int router_mode,
-                                                     float* __restrict__ tok_out, uint64_t* stamp) {
+                                                     float* __restrict__ tok_out, int cap_max, uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     // One pass: the row stays in registers between the sum of squares and the scaling
     // (up to kMaxV float4 per thread; longer rows re-read the tail from L1/L2).
@@ -102,12 +102,14 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
     pdl_wait();
     __shared__ float red[32];
     __shared__ float red_r[32];
+    // cap_max: the context was sized for slabs of at most this many tokens (the attention grid covers no more);
+    // a longer slab is used up to there and then counts as full
     if (len_inc && threadIdx.x == 0) {
         const int T = len_inc[b];
-        if (T < slab_cap[b]) len_inc[b] = T + 1;
+        if (T < min(slab_cap[b], cap_max)) len_inc[b] = T + 1;
     }
     if (rowinfo && threadIdx.x == (blockDim.x > 32 ? 32 : 0)) {
-        const int T = len_ro[b], cap = slab_cap[b];
+        const int T = len_ro[b], cap = min(slab_cap[b], cap_max);
         const bool room = T < cap;
         rowinfo[i] = make_longlong2((long long)min(T + 1, cap) | ((long long)b << 32),
                                     (long long)slab_off[b] | (room ? (1ll << 62) : 0ll));
@@ -185,7 +187,8 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                                                   const int64_t* __restrict__ slab_off,
                                                   const int32_t* __restrict__ slab_cap,
                                                   const int32_t* len_l, uint32_t* __restrict__ flags,
-                                                  longlong2* __restrict__ rowinfo, int pair, uint64_t* stamp) {
+                                                  longlong2* __restrict__ rowinfo, int pair, int cap_max,
+                                                  uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     pdl_trigger();
     const int m = m_dev ? min((int)gridDim.y, __ldg(m_dev)) : (int)gridDim.y;
@@ -203,12 +206,12 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                 const int b0 = idx[i0], b1 = idx[i0 + 1];
                 const int t0 = len_l[b0];
                 return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == t0 + 1 &&
-                       t0 + 1 < slab_cap[b1] && !(t0 & 1);
+                       t0 + 1 < min(slab_cap[b1], cap_max) && !(t0 & 1);
             };
             if (is_pair(i - 1)) y |= 1ll << 60;
             else if (is_pair(i)) y |= 1ll << 61;
         }
-        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, slab_cap[b]) | ((long long)b << 32), y);
+        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, min(slab_cap[b], cap_max)) | ((long long)b << 32), y);
     }
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
         return;
     }
     const int T = len_l[b];
-    if (T >= slab_cap[b]) {
+    if (T >= min(slab_cap[b], cap_max)) {  // (a slab longer than the context was sized for is full at that size)
         if (head == Hq && d == 0) atomicOr(flags, FIRST_FLAG_KV_FULL);
         return;
     }

@@ -251,11 +251,26 @@ def test_decode_bf16_gqa_ragged(shape):
 @pytest.mark.parametrize("B", [70, 200, 300])
 def test_decode_bf16_many_rows(B):
     """Many active rows: wide activation tiles (one projection CTA per SM), and with 300 rows more than one
-    256-row projection launch per matrix."""
+    256-row projection launch per matrix.  Once with the default kernels (CTA pairs from 96 rows on), once with
+    the single-CTA kernel at every size."""
     shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
     lens = fi.prompt_lengths(B, 1, 90, 13)
     mask = fi.mask_bernoulli(B, shape.n_layers, 0.85, 14)
     errs, agrees = _run_decode_case(shape, True, lens, mask, 2, 16, 2e-2)
+    assert agrees.mean() >= 0.98
+    errs, agrees = _run_decode_case(shape, True, lens, mask, 2, 16, 2e-2, options={"tc2_min_rows": 0})
+    assert agrees.mean() >= 0.98
+
+
+@pytest.mark.parametrize("B", [100, 40, 130, 200, 256, 300])
+def test_decode_bf16_cta_pair_projections(B):
+    """The CTA-pair projection kernel (two CTAs per tile pair, activation rows split between them), forced from 33
+    rows on: 33..64 rows (one 16-row group per CTA and a ragged second), 100, 130, 200, 256 rows, and 300 rows
+    (a 256-row launch plus a 44-row launch per matrix)."""
+    shape = fi.ModelShape(2, 512, 8, 2, 128, 1024, 1000, 500000.0)
+    lens = fi.prompt_lengths(B, 1, 90, 13)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.85, 14)
+    errs, agrees = _run_decode_case(shape, True, lens, mask, 2, 16, 2e-2, options={"tc2_min_rows": 33})
     assert agrees.mean() >= 0.98
 
 
@@ -408,6 +423,34 @@ def test_full_slab_on_the_tuned_attention_path():
     ref = oracle.decode_step(om, toks[1:2], np.ones((1, shape.n_layers), np.uint8), solo)
     err, _ = logits_check(logits[1:2].cpu().numpy(), ref)
     assert err.max() <= 2e-2
+
+
+@pytest.mark.parametrize("options", [None, {"fuse_rope": 0}, {"attn_simple": 1}])
+def test_slab_longer_than_the_context_was_sized_for_is_full_at_that_size(options):
+    """slab_cap may exceed max_tokens_per_seq (the caller's table, never checked on the host): such a slab is used
+    up to max_tokens_per_seq and then counts as full -- flag raised, cache and length untouched -- instead of
+    outrunning the attention launch, which is sized by max_tokens_per_seq."""
+    import torch
+    shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
+    w = fi.make_weights(shape, 2, True)
+    MAXT = 70
+    okv, gkv = synthetic_caches(shape, [70, 40], [70 + 64, 60], 1, True)   # slab 0: 134 rows, 70 present
+    ctx = _ctx(shape, True, 2, MAXT, w)
+    for k, v in (options or {}).items():
+        ctx.set_option(k, v)
+    ctx.set_mask(torch.ones((2, shape.n_layers), dtype=torch.uint8, device="cuda"))
+    before = [gkv.rows_host(l, 0) for l in range(shape.n_layers)]
+    logits = torch.empty((2, shape.vocab), dtype=torch.float32, device="cuda")
+    toks = fi.tokens(shape, 2, 5, "t")
+    for step in range(2):
+        ctx.decode_step(torch.from_numpy(toks).cuda(), gkv.c, logits)
+        assert ctx.device_flags() == 1  # FIRST_FLAG_KV_FULL, every step
+    for l in range(shape.n_layers):
+        k1, v1 = gkv.rows_host(l, 0)
+        assert np.array_equal(k1, before[l][0]) and np.array_equal(v1, before[l][1])
+    assert gkv.len.cpu().numpy()[:, 0].tolist() == [70] * shape.n_layers
+    assert gkv.len.cpu().numpy()[:, 1].tolist() == [42] * shape.n_layers
+    assert np.isfinite(logits.cpu().numpy()).all()
 
 
 def test_a_wait_that_runs_out_raises_the_flag_and_the_context_stays_usable():
