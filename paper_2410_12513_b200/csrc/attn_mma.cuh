@@ -74,7 +74,12 @@ struct RopeFuse {
 // and value already in the slab); bit 60 = row i is served by row i-1 (its CTAs exit).  The second row's query
 // heads take fragment rows G..2G-1 (so 2G <= 8), share every K/V tile with the first row's, and see one token
 // more at the end.  Not combined with RopeFuse.
-template <int HD, int G, bool PAIR = false>
+// CL (decode only): the grid is launched as thread-block clusters of gridDim.x CTAs, one cluster per (row, kv head),
+// and a split row's chunks meet in the shared memory of the cluster's first CTA instead of in global memory: every
+// other chunk writes its partial result there (distributed shared memory, plain remote stores -- no multicast load
+// anywhere), arrives at the cluster barrier and leaves; the first CTA waits at that barrier and merges.  No global
+// round trip, no fence, no ticket.  Needs (gridDim.x - 1) * GR * (HD + 2) floats of shared memory behind the ring.
+template <int HD, int G, bool PAIR = false, bool CL = false>
 __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV,
                                                       const float* q, int64_t cap_total,
@@ -334,6 +339,16 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
     float* o_s = reinterpret_cast<float*>(base_ptr);       // [4][GR][HD]
     float* m_s = o_s + 4 * GR * HD;                         // [4][GR]
     float* l_s = m_s + 4 * GR;                              // [4][GR]
+    // CL: behind the ring, never touched by a copy: [S_max-1][GR][HD+2] partials of chunks 1.. (written by them,
+    // remotely), then this CTA's own partial [GR][HD] and its (max, sum) [2][GR]
+    float* part_s = reinterpret_cast<float*>(base_ptr + kStages * kStageBytes);
+    float* part0_s = part_s + (gridDim.x - 1) * GR * (HD + 2);
+    float* ml0_s = part0_s + GR * HD;
+    uint32_t part_remote = 0;
+    if (CL) {
+        const uint32_t local = base + (uint32_t)(kStages * kStageBytes);
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(part_remote) : "r"(local), "r"(0));
+    }
     if (g < GR) {
 #pragma unroll
         for (int nt = 0; nt < kNTiles; ++nt) {
@@ -369,12 +384,58 @@ __global__ void __launch_bounds__(160) attn_split_mma(const __grid_constant__ CU
         }
         if (n_chunks == 1) {
             emit(hq_of(gg), d, acc / l);  // the whole row in one chunk: done
+        } else if (CL) {
+            if (c == 0) {  // the merging CTA keeps its own partial in registers-to-shared form
+                part0_s[gg * HD + d] = acc;
+                if (d == 0) { ml0_s[gg] = M; ml0_s[GR + gg] = l; }
+            } else {       // chunk c > 0: slot c-1 of the first CTA's buffer
+                const uint32_t slot = part_remote + (uint32_t)(((c - 1) * GR + gg) * (HD + 2)) * 4u;
+                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(slot + (uint32_t)d * 4u), "f"(acc) : "memory");
+                if (d == 0) {
+                    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(slot + (uint32_t)HD * 4u), "f"(M) : "memory");
+                    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(slot + (uint32_t)(HD + 1) * 4u), "f"(l) : "memory");
+                }
+            }
         } else {
             o_part[(hq_of(gg) * S_max + c) * HD + d] = acc;
             if (d == 0) ml_part[hq_of(gg) * S_max + c] = make_float2(M, l);
         }
     }
     if (n_chunks == 1) return;
+    if (CL) {
+        // Every consumer thread of every live chunk arrives (release: its remote stores are visible to whoever
+        // acquires); chunks other than the first leave at once.  Threads that have exited (producer warps, work items
+        // past the row's end) are not waited for.
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (c != 0) return;
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        bar_consumers();  // part0_s / ml0_s of all four warps
+        float* w_s = o_s;  // [2][GR][64], as below; o_s is free again
+        for (int e = threadIdx.x; e < rows_live * n_chunks; e += kConsumers) {
+            const int gg = e / n_chunks, sidx = e - gg * n_chunks;
+            const float* src = sidx == 0 ? nullptr : part_s + ((sidx - 1) * GR + gg) * (HD + 2) + HD;
+            w_s[gg * 64 + sidx] = sidx == 0 ? ml0_s[gg] : src[0];
+            w_s[(GR + gg) * 64 + sidx] = sidx == 0 ? ml0_s[GR + gg] : src[1];
+        }
+        bar_consumers();
+        if (threadIdx.x < rows_live) {
+            const int gg = threadIdx.x;
+            float M = -INFINITY, den = 0.f;
+            for (int sidx = 0; sidx < n_chunks; ++sidx) M = fmaxf(M, w_s[gg * 64 + sidx]);
+            for (int sidx = 0; sidx < n_chunks; ++sidx) den += w_s[(GR + gg) * 64 + sidx] * __expf(w_s[gg * 64 + sidx] - M);
+            const float inv = 1.f / den;
+            for (int sidx = 0; sidx < n_chunks; ++sidx) w_s[gg * 64 + sidx] = __expf(w_s[gg * 64 + sidx] - M) * inv;
+        }
+        bar_consumers();
+        for (int e = threadIdx.x; e < rows_live * HD; e += kConsumers) {
+            const int gg = e / HD, d = e - gg * HD;
+            const float* wv = w_s + gg * 64;
+            float acc = part0_s[gg * HD + d] * wv[0];
+            for (int sidx = 1; sidx < n_chunks; ++sidx) acc += part_s[((sidx - 1) * GR + gg) * (HD + 2) + d] * wv[sidx];
+            emit(hq_of(gg), d, acc);
+        }
+        return;
+    }
     // ---- ticket: the last chunk of this (row, kv head) to get here merges them all
     __threadfence();
     bar_consumers();

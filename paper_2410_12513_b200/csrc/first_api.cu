@@ -97,6 +97,7 @@ struct first_ctx {
     int stamp_n = 0;
     std::vector<int> stamp_cls;
     // options
+    int attn_cluster = 0;   // split attention rows merge through a thread-block cluster's shared memory
     int tc2_min_rows = 96;  // from this many rows on a projection launch uses the CTA-pair kernel (0 = never)
     int tc2_mt2_all = 0;    // CTA-pair kernel: two weight tiles per unit for the reducing epilogues too
     int max_gemv_rows = -1;
@@ -572,6 +573,37 @@ int launch_attn_mma_hg(first_ctx* c, cudaStream_t st, dim3 grid, const CUtensorM
         rf.k_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(kc));
         rf.v_slab = static_cast<__nv_bfloat16*>(const_cast<void*>(vc));
     }
+    // Split rows: the chunks of a (row, kv head) form a thread-block cluster and merge through the first CTA's shared
+    // memory when the cluster is small enough (at most 8 CTAs) and its partial results fit beside the ring without
+    // costing the second CTA per SM.
+    constexpr int GR = G;
+    const int S = (int)grid.x;
+    const int part_bytes = ((S - 1) * GR * (HD + 2) + GR * HD + 2 * GR) * 4;
+    if (!PAIR && c->attn_cluster && S > 1 && S <= 8 && smem + part_bytes <= 113 * 1024) {
+        if constexpr (!PAIR) {
+            Launch guard(c, st, kClsAttn);
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = grid;
+            cfg.blockDim = dim3(160);
+            cfg.dynamicSmemBytes = smem + part_bytes;
+            cfg.stream = st;
+            cudaLaunchAttribute at[2];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = S;
+            at[0].val.clusterDim.y = 1;
+            at[0].val.clusterDim.z = 1;
+            at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            at[1].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = at;
+            cfg.numAttrs = (c->use_pdl && !c->profiling && c->pdl_next) ? 2 : 1;
+            c->pdl_next = true;
+            uint64_t* stamp = stamp_slot(c, kClsAttn);
+            CU_TRY(cudaLaunchKernelEx(&cfg, attn::attn_split_mma<HD, G, false, true>, tk, tv, (const float*)c->q, kv->cap_total,
+                                      (const longlong2*)c->rowinfo, m_dev, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket,
+                                      out, out_hi, out_lo, c->flags, rf, stamp));
+            return FIRST_OK;
+        }
+    }
     return launch_k(c, st, kClsAttn, attn::attn_split_mma<HD, G, PAIR>, grid, dim3(160), smem, tk, tv, c->q, kv->cap_total,
                     c->rowinfo, m_dev, c->d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out,
                     out_hi, out_lo, c->flags, rf);
@@ -581,6 +613,7 @@ template <int HD, int G>
 int attn_mma_set_attr() {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024));
     if constexpr (2 * G <= 8)  // the two-rows-per-work-item form used on prompt chunks
         CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     return FIRST_OK;
@@ -1299,6 +1332,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc_smem_kb")) c->tc_smem_kb = value > 0 ? (int)value : 110;
     else if (!std::strcmp(name, "tc2_min_rows")) c->tc2_min_rows = value < 0 ? 96 : (int)value;
     else if (!std::strcmp(name, "tc2_mt2_all")) c->tc2_mt2_all = value > 0;
+    else if (!std::strcmp(name, "attn_cluster")) c->attn_cluster = value > 0;
     else if (!std::strcmp(name, "stamp")) {
         c->stamp_on = value > 0;
         if (c->stamp_on && !c->stamps) {

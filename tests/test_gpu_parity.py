@@ -274,6 +274,20 @@ def test_decode_bf16_cta_pair_projections(B):
     assert agrees.mean() >= 0.98
 
 
+@pytest.mark.parametrize("hq,hkv,hd", [(8, 2, 128), (8, 2, 64), (6, 2, 128), (8, 1, 64), (4, 4, 128)])
+def test_decode_bf16_split_rows_merged_through_a_cluster(hq, hkv, hd):
+    """Rows long enough to be split into several attention chunks, with the chunks of a (row, kv head) merged through
+    the shared memory of a thread-block cluster (option attn_cluster) and, for comparison, through global memory:
+    1 to 5 chunks per row (chunks of 64 tokens), rows of one token, a full slab among them."""
+    shape = fi.ModelShape(2, hq * hd // 2 if hq * hd // 2 >= 256 else 256, hq, hkv, hd, 512, 1000, 500000.0)
+    lens = np.array([300, 1, 64, 65, 129, 200, 17, 256], np.int32)
+    mask = fi.mask_bernoulli(len(lens), shape.n_layers, 0.8, 4)
+    for opts in ({"attn_chunk": 64, "attn_cluster": 1}, {"attn_chunk": 64, "attn_cluster": 0},
+                 {"attn_chunk": 128, "attn_cluster": 1}):
+        errs, agrees = _run_decode_case(shape, True, lens, mask, 3, 6, 2e-2, options=opts)
+        assert agrees.mean() >= 0.9
+
+
 def test_decode_bf16_gemv_path_and_general_attention_by_option():
     """The CUDA-core GEMV projections and the general attention kernel, forced by option, on a bf16 model."""
     shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
