@@ -472,6 +472,25 @@ class Job:
         ms = max_over_ranks(e0.elapsed_time(e1), self.dist, self.dist_dev)
         return ms, self.ctx.launch_count() - l0
 
+    def step_percentiles(self, mask, n=48, W=5):
+        """Per-step latency: an event after every step of an untimed run (the events add nothing to a step that is one
+        graph launch); p10 / p50 / p90 in ms."""
+        torch = self.torch
+        self.ctx.set_mask(torch.from_numpy(np.ascontiguousarray(mask)).to(self.dev))
+        self.reset()
+        self.steps(W)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        a, b = self.tok_a, self.tok_b
+        ev[0].record(self.stream)
+        for i in range(n):
+            self.ctx.decode_step(a, self.kv, None, b)
+            a, b = b, a
+            ev[i + 1].record(self.stream)
+        torch.cuda.synchronize()
+        t = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(n)])
+        return {"p10": float(np.percentile(t, 10)), "p50": float(np.percentile(t, 50)), "p90": float(np.percentile(t, 90)),
+                "steps": n}
+
     def in_step_ms(self, mask, n=8):
         """Where a step's time goes while it runs the way it is timed (one graph, dependent launches overlapping):
         every launch stamps first-CTA start / last-warp end; per class, the time from the previous launch's end to
@@ -664,6 +683,7 @@ def run_cuda(args, wl, shape, mask, lens):
     e2e = {"value": job_tokens_per_s(world, B, K, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": B * 4,
            "d2h_bytes_per_step": B * 4, "ms_per_step": e2e_ms / K}
 
+    pct = job.step_percentiles(mask, n=min(48, K), W=W)
     # ---- where the step's time goes: in-step stamps (nothing serialised), then event pairs (serialised)
     excl_ms, span_ms, cls_launches, traced_step_ms = job.in_step_ms(mask)
     ctx.set_mask(torch.from_numpy(mask).to(dev))
@@ -734,7 +754,7 @@ def run_cuda(args, wl, shape, mask, lens):
            "dense": {"ms_per_step": dense_ms, "gpu_launches": int(dense_launches), "bytes_strict": bm_dense["strict"],
                      "latency_ratio_routed_over_dense": ms_step / dense_ms,
                      "bytes_ratio_routed_over_dense": bm["full"] / bm_dense["full"]},
-           "ms_per_step_repeat": repeat_ms, "skip_sweep": sweep,
+           "ms_per_step_repeat": repeat_ms, "step_latency_ms": pct, "skip_sweep": sweep,
            "kernel_ms_in_step": in_step, "traced_step_ms": traced_step_ms,
            "kernel_ms_per_step_event_pairs": cls_ms, "route": route}
     if not args.no_join and rank == 0:

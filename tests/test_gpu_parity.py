@@ -776,6 +776,46 @@ def test_per_layer_slab_tables(bf16):
     assert torch.equal(kv2.len, gkv.len) and torch.equal(kv2.pos, gkv.pos)
 
 
+def test_in_step_trace_lists_every_launch_in_order():
+    """Option "stamp": every launch of a step records first-CTA start and last-warp end; the trace has one entry
+    per launch, in launch order, with start <= end, ends non-decreasing along the dependency chain, and the logits
+    are the same as without it."""
+    import torch
+    shape = fi.ModelShape(3, 256, 8, 2, 64, 512, 1000, 500000.0)
+    B = 6
+    w = fi.make_weights(shape, 3, True)
+    lens = fi.prompt_lengths(B, 1, 100, 3)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.7, 4)
+    mask[:, 1] = 0                                   # a layer nobody keeps: no launches for it
+    okv, gkv = synthetic_caches(shape, lens, [int(n) + 4 for n in lens], 3, True)
+    ctx = _ctx(shape, True, B, int(max(lens)) + 4, w)
+    ctx.set_mask(torch.from_numpy(mask).cuda())
+    toks = torch.from_numpy(fi.tokens(shape, B, 3, "first")).cuda()
+    logits = torch.empty((B, shape.vocab), dtype=torch.float32, device="cuda")
+    l0 = ctx.launch_count()
+    ctx.decode_step(toks, gkv.c, logits)
+    per_step = ctx.launch_count() - l0
+    plain = logits.cpu().numpy().copy()
+    gkv.set_len(okv.len, okv.pos)
+    ctx.set_option("stamp", 1)
+    ctx.decode_step(toks, gkv.c, logits)
+    tr = ctx.step_trace()
+    assert len(tr) == per_step == 1 + 7 * 2 + 3      # begin, 7 per kept layer, final norm + lm_head + end
+    names = [t[0] for t in tr]
+    assert names[0] == "step_begin" and names[-1] == "step_end" and names.count("attn_split") == 2
+    assert names.count("rmsnorm_rows") == 5 and names.count("gemm_tc") == 9
+    assert all(0 < t0 <= t1 for _, t0, t1 in tr)
+    ends = [t1 for _, _, t1 in tr]
+    assert all(b >= a for a, b in zip(ends, ends[1:]))   # each kernel ends after the one it depends on
+    assert (ends[-1] - tr[0][1]) < 50_000_000            # one clock, nanoseconds: the step took well under 50 ms
+    err, _ = logits_check(logits.cpu().numpy(), plain)
+    assert err.max() <= 1e-3                               # same step (float32 reduction order may differ)
+    ctx.set_option("stamp", 0)
+    with pytest.raises(Exception):
+        ctx.step_trace()
+    assert ctx.device_flags() == 0
+
+
 def test_documented_error_statuses():
     """The statuses the header promises: unsupported shapes at create, call order, capacity, sampling limits."""
     import dataclasses
