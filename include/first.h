@@ -415,6 +415,9 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *                    itself, from the QKV projection's output.
  *   "prefill_pair"   0 = in first_prefill every prompt token has attention work items of its own.  Default 1:
  *                    two consecutive tokens of a sequence share them (up to 4 query heads per KV head).
+ *   "prefill_group"  0 = no groups.  Default 1: in first_prefill up to eight consecutive tokens of a sequence (one
+ *                    block of eight positions) share attention work items, so a prefix's keys/values are staged once
+ *                    per eight tokens (up to 4 query heads per KV head; otherwise the pair form or single rows)
  *   "prefill_rows"   prompt tokens per chunk of first_prefill, 1..256 (default 256; never more than max_batch)
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in

@@ -9,6 +9,7 @@
 #include <unordered_map>
 
 #include "attn_mma.cuh"
+#include "attn_prefill.cuh"
 #include "attn_simple.cuh"
 #include "common.cuh"
 #include "first.h"
@@ -106,6 +107,7 @@ struct first_ctx {
     int fuse_swiglu = 1;
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
+    int prefill_group = 1; // prompt chunks: up to eight consecutive tokens share one (takes precedence over pairs)
     int prefill_rows = 0;  // rows per prompt chunk (0: 256)
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
@@ -614,6 +616,8 @@ int attn_mma_set_attr() {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024));
+    if constexpr (2 * G <= 8)  // the group form used on prompt chunks
+        CU_TRY(cudaFuncSetAttribute(attn::attn_group_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     if constexpr (2 * G <= 8)  // the two-rows-per-work-item form used on prompt chunks
         CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     return FIRST_OK;
@@ -632,7 +636,7 @@ int attn_mma_setup(first_ctx* c) {
 // Tuned attention for bfloat16 caches with head_dim 64/128; returns FIRST_E_UNSUPPORTED otherwise.
 int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const void* vc, const LayerKv* kv,
                     const int32_t* len_l, const int32_t* idx, float* out, __nv_bfloat16* out_hi,
-                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, bool pair, const int32_t* m_dev) {
+                    __nv_bfloat16* out_lo, bool fuse_rope, float qscale, int pair, const int32_t* m_dev) {
     const first_model_desc& d = c->d;
     if ((uint64_t)d.n_kv_heads * (uint64_t)kv->cap_total >= (1ull << 31)) return FIRST_E_UNSUPPORTED;
     int C = c->attn_chunk;
@@ -652,6 +656,16 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     int rc;
     if ((rc = kv_map_for(c, kc, kv->cap_total, &tk)) || (rc = kv_map_for(c, vc, kv->cap_total, &tv))) return rc;
     dim3 grid(S, d.n_kv_heads, m);
+#define FIRST_ATTN_GROUP(HD, G)                                                                                  \
+    if (pair == 2 && d.head_dim == HD && c->group == G) {                                                        \
+        constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;                           \
+        return launch_k(c, st, kClsAttn, attn::attn_group_mma<HD, G>, dim3(grid.x, grid.y, (m + 7) / 8),         \
+                        dim3(160), smem, *tk, *tv, c->q, kv->cap_total, c->rowinfo, m, m_dev, d.n_q_heads, C,    \
+                        c->o_part, c->ml_part, c->ticket, out, out_hi, out_lo, c->flags);                        \
+    }
+    FIRST_ATTN_GROUP(128, 1) FIRST_ATTN_GROUP(128, 2) FIRST_ATTN_GROUP(128, 3) FIRST_ATTN_GROUP(128, 4)
+    FIRST_ATTN_GROUP(64, 1) FIRST_ATTN_GROUP(64, 2) FIRST_ATTN_GROUP(64, 3) FIRST_ATTN_GROUP(64, 4)
+#undef FIRST_ATTN_GROUP
 #define FIRST_ATTN_PAIR(HD, G)                            \
     if (pair && d.head_dim == HD && c->group == G)        \
         return launch_attn_mma_hg<HD, G, true>(c, st, grid, *tk, *tv, kv, kc, vc, C, out, out_hi, out_lo, false, qscale, m_dev);
@@ -716,7 +730,8 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     const bool fuse_rope = mma_attn && c->fuse_rope;
     // prompt chunks: consecutive rows are consecutive tokens of a sequence and may share attention work items
     const bool route_here = ph && ph->router_w;
-    const bool pair_rows = ph && mma_attn && !fuse_rope && c->prefill_pair && 2 * c->group <= 8;
+    // (0 = each row its own work items, 1 = pairs of consecutive tokens, 2 = groups of up to eight)
+    const int pair_rows = (ph && mma_attn && !fuse_rope && 2 * c->group <= 8) ? (c->prefill_group ? 2 : c->prefill_pair ? 1 : 0) : 0;
 
     for (int l = 0; l < L; ++l) {
         if (layer_inputs) {
@@ -757,7 +772,7 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
             (rc = launch_k(c, st, kClsRopeAppend, rope_append<WT>, dim3((d.n_q_heads + 2 * d.n_kv_heads + 7) / 8, m), dim3(hd / 2, 8),
                            0, c->qkv, idx, m_dev, d.n_q_heads, d.n_kv_heads, hd, c->cs, qscale, c->q,
                            static_cast<WT*>(kv->k[l]), static_cast<WT*>(kv->v[l]), lkv.cap_total, lkv.slab_off,
-                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows ? 1 : 0,
+                           lkv.slab_cap, len_l, c->flags, mma_attn ? c->rowinfo : nullptr, pair_rows,
                            d.max_tokens_per_seq)))
             return rc;
         if (mma_attn) {
@@ -1325,6 +1340,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "fuse_swiglu")) c->fuse_swiglu = value != 0;
     else if (!std::strcmp(name, "fuse_rope")) c->fuse_rope = value != 0;
     else if (!std::strcmp(name, "prefill_pair")) c->prefill_pair = value != 0;
+    else if (!std::strcmp(name, "prefill_group")) c->prefill_group = value != 0;
     else if (!std::strcmp(name, "prefill_rows")) c->prefill_rows = value > 0 ? (int)value : 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;

@@ -177,6 +177,8 @@ __global__ void __launch_bounds__(1024) rmsnorm_rows(const float* x, const int32
 // (hd/2, 8): eight heads of a row per block; thread (d, .) handles the rotary pair (d, d+hd/2) of its head.
 // len is only read here (the FFN-side rmsnorm_rows advances it once attention is done).
 // rowinfo[i] = (tokens to attend over, first slab row) saves the attention CTAs two dependent loads.
+// pair: 0 = every row has work items of its own; 1 = mark pairs of consecutive tokens (attn_split_mma's pair form);
+// 2 = mark groups of up to eight consecutive tokens (attn_group_mma).
 // A full slab sets FIRST_FLAG_KV_FULL and leaves the cache alone.
 template <typename KT>
 __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32_t* __restrict__ idx,
@@ -208,8 +210,28 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                 return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == t0 + 1 &&
                        t0 + 1 < min(slab_cap[b1], cap_max) && !(t0 & 1);
             };
-            if (is_pair(i - 1)) y |= 1ll << 60;
-            else if (is_pair(i)) y |= 1ll << 61;
+            if (pair == 1) {
+                if (is_pair(i - 1)) y |= 1ll << 60;
+                else if (is_pair(i)) y |= 1ll << 61;
+            } else {
+                // Groups (attn_group_mma): up to eight consecutive tokens of one slab inside one block of eight
+                // positions.  A row leads a group unless it continues its predecessor's (again a local rule): bit 60
+                // = served by the leader; a leader carries its member count - 1 in bits 56..59.
+                auto consec = [&](int a) {  // rows a, a+1: consecutive tokens of one slab, the second with room
+                    if (a < 0 || a + 1 >= m) return false;
+                    const int b0 = idx[a], b1 = idx[a + 1];
+                    return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == len_l[b0] + 1 &&
+                           len_l[b1] < min(slab_cap[b1], cap_max);
+                };
+                const int p = len_l[b];
+                if (consec(i - 1) && (p & 7) != 0) {
+                    y |= 1ll << 60;
+                } else {
+                    int n = 1;
+                    while (n < 8 && ((p + n) & 7) != 0 && consec(i + n - 1)) ++n;
+                    y |= (long long)(n - 1) << 56;
+                }
+            }
         }
         rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, min(slab_cap[b], cap_max)) | ((long long)b << 32), y);
     }

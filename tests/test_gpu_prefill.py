@@ -132,7 +132,24 @@ def test_prefill_bf16_query_head_groupings(hq, hkv, hd):
 
 
 def test_prefill_bf16_pairing_off_by_option():
-    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"prefill_pair": 0, "prefill_rows": 20})
+    """Every prompt token with attention work items of its own (neither groups of eight nor pairs)."""
+    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2,
+                  {"prefill_group": 0, "prefill_pair": 0, "prefill_rows": 20})
+
+
+def test_prefill_bf16_pairs_by_option():
+    """The pair form (two consecutive tokens per work item), which groups of eight replaced as the default."""
+    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"prefill_group": 0, "prefill_rows": 20})
+    _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 200], 256, 2, 7, 0, 0.6, 2e-2, {"prefill_group": 0})
+
+
+@pytest.mark.parametrize("rows,chunk_tokens", [(20, 64), (256, 64), (37, 128), (256, 1024)])
+def test_prefill_bf16_groups_of_eight(rows, chunk_tokens):
+    """Groups of up to eight consecutive tokens per attention work item (the default), at chunk heights that cut
+    groups at odd places (20, 37 rows), with prompts of 1, 2, 7, 8, 9 tokens (groups of every size, sequences that
+    start in the middle of a chunk) and prompts long enough for several token chunks per group (merged by ticket)."""
+    _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 7, 8, 9, 300, 16], rows, 2, 8, 1, 0.6, 2e-2,
+                  {"prefill_rows": rows, "attn_chunk": chunk_tokens})
 
 
 def test_prefill_bf16_general_kernels_by_option():
