@@ -403,6 +403,7 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *   "tc_mt2_min_rows" from this many active rows on a projection CTA takes two weight tiles per
  *                    activation tile (default: when the activation tiles are so wide that only one
  *                    single-tile CTA would fit per SM, i.e. from 96 rows)
+ *   "norm_threads"   threads per RMSNorm CTA (one CTA per row), a multiple of 32 up to 1024; default 512
  *   "attn_cluster"   1 = the chunks of a split attention row are launched as a thread-block cluster and merge through
  *                    the first chunk's shared memory (up to 8 chunks) instead of through global memory; default 0
  *   "tc2_min_rows"   from this many active rows on a tensor-core projection launch runs as CTA pairs (two SMs per
