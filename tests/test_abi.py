@@ -35,6 +35,20 @@ def test_status_strings_and_null_argument_errors_need_no_gpu():
     assert L.first_prefill_route(None, 0, None, 0, None, 1, 1, None, None, 0.5, 0, None, None, None) == -1
     assert L.first_prefill(None, None, None, 1, None, None, None, 0.5, 0, None, None, None, None, None) == -1
     assert L.first_destroy(None) == 0
+    # the entry points for changing batches and the measurement aids reject missing arguments the same way
+    assert L.first_set_mask_host(None, None, 1, None) == -1
+    assert L.first_pool_create(None, 4, None, None, None, None) == -1
+    assert L.first_seq_join(None, None, 8, None, 0, 0, None, None) == -1
+    assert L.first_seq_leave(None, 0, None) == -1
+    assert L.first_pool_commit(None, None) == -1
+    assert L.first_pool_kv(None, None) == -1
+    assert L.first_pool_stats(None, None, None, None) == -1
+    assert L.first_pool_destroy(None) == 0
+    assert L.first_step_trace(None, 0, None, None, None, None, None) == -1
+    assert L.first_selftest_wait_expiry(None, 10, None, None, None) == -1
+    assert L.first_graph_count(None) == 0
+    assert {"first_pool_create", "first_seq_join", "first_seq_leave", "first_pool_commit", "first_set_mask_host",
+            "first_step_trace", "first_prefill_route_static"} <= set(_declared())
 
 
 def test_product_package_does_not_import_the_oracle():
