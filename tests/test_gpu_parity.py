@@ -288,6 +288,19 @@ def test_decode_bf16_split_rows_merged_through_a_cluster(hq, hkv, hd):
         assert agrees.mean() >= 0.9
 
 
+@pytest.mark.parametrize("ffn", [320, 352, 448])
+def test_decode_bf16_many_rows_with_ragged_feature_counts(ffn):
+    """120-150 active rows (CTA-pair projections) on widths that do not fill the last weight tile: FFN widths that
+    are a multiple of 64 but not of 256 (fused SwiGLU falls back to the single-CTA kernel), or not even of 64 (gate/up
+    as a plain reducing projection through the CTA pairs + the separate activation kernel), vocabulary 1000."""
+    shape = fi.ModelShape(2, 320, 5, 5, 64, ffn, 1000, 500000.0)
+    B = 150
+    lens = fi.prompt_lengths(B, 1, 70, 17)
+    mask = fi.mask_bernoulli(B, shape.n_layers, 0.85, 18)
+    errs, agrees = _run_decode_case(shape, True, lens, mask, 2, 19, 2e-2)
+    assert agrees.mean() >= 0.98
+
+
 def test_decode_bf16_gemv_path_and_general_attention_by_option():
     """The CUDA-core GEMV projections and the general attention kernel, forced by option, on a bf16 model."""
     shape = fi.ModelShape(2, 256, 8, 2, 128, 512, 1000, 500000.0)
