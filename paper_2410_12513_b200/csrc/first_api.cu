@@ -98,7 +98,6 @@ struct first_ctx {
     int stamp_n = 0;
     std::vector<int> stamp_cls;
     // options
-    int tc_pf_ahead = 0;          // single-CTA projections: L2 look-ahead of the weight stream, in k-blocks
     int norm_threads_max = 512;   // threads per norm CTA (one row each): 512 measured 8 % faster in-step than 1024 at D = 4096
     int attn_cluster = 0;   // split attention rows merge through a thread-block cluster's shared memory
     int tc2_min_rows = 96;  // from this many rows on a projection launch uses the CTA-pair kernel (0 = never)
@@ -435,7 +434,6 @@ int launch_gemm_tc(first_ctx* c, cudaStream_t st, const CUtensorMap& tmA, const 
         p.stamp = stamp_slot(c, kClsGemmTc);
         p.m_dev = m_dev;
         p.row0 = r0;
-        p.pf_ahead = c->tc_pf_ahead;
         CUtensorMap tmBh, tmBl;
         if ((rc = make_map(&tmBh, Xh + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
         if ((rc = make_map(&tmBl, Xl + (size_t)r0 * K, mm, K, p.n_pad, false))) return rc;
@@ -1352,7 +1350,6 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "tc2_min_rows")) c->tc2_min_rows = value < 0 ? 96 : (int)value;
     else if (!std::strcmp(name, "tc2_mt2_all")) c->tc2_mt2_all = value > 0;
     else if (!std::strcmp(name, "attn_cluster")) c->attn_cluster = value > 0;
-    else if (!std::strcmp(name, "tc_pf_ahead")) c->tc_pf_ahead = value > 0 ? std::min<int>((int)value, 32) : 0;
     else if (!std::strcmp(name, "norm_threads")) c->norm_threads_max = value >= 32 ? std::min<int>(1024, (int)value / 32 * 32) : 512;
     else if (!std::strcmp(name, "stamp")) {
         c->stamp_on = value > 0;

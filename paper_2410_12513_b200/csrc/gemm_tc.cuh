@@ -51,7 +51,6 @@ struct GemmParams {
     __nv_bfloat16* act_hi;   // [m][n_out] bfloat16 hi/lo split or NULL
     __nv_bfloat16* act_lo;
     uint64_t* stamp;         // in-step timing slot or NULL
-    int pf_ahead;            // weight tiles asked into L2 this many k-blocks ahead of the ring (0 = off)
     const int32_t* m_dev;    // active-row count in device memory (m is a host-side upper bound of it) or NULL
     int row0;                // first compact row of this launch (launches take 256 rows each)
 };
@@ -95,12 +94,6 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
         "[%0], [%1, {%3, %4}], [%2], %5;"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
-}
-
-// Ask for a tile to be brought into L2 (no shared memory, no barrier): used to look further ahead in a CTA's own
-// weight stream than its shared-memory ring reaches.
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
 }
 
 // Shared-memory matrix descriptor, K-major operand in 128-byte-swizzled rows:
@@ -181,19 +174,6 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
                 tma_load_2d_hint(sa + a * kABytes, &tmA, bar, kc, (tile * p.mt + a) * kBlockM, pol_stream);
         }
     };
-    // k-block i of this CTA's weight tiles -> L2 (look-ahead beyond the ring; p.pf_ahead k-blocks, 0 = off)
-    auto prefetch_a = [&](int i) {
-        if (i >= nkb) return;
-        const int kc = (kb0 + i) * kBlockK;
-        if (EPI == kEpiSwiglu) {
-            const int rows = p.mt == 1 ? p.pair_rows : 128;
-            const CUtensorMap* tm = p.mt == 1 ? &tmA : &tmA2;
-            tma_prefetch_2d(tm, kc, tile * rows);
-            tma_prefetch_2d(tm, kc, p.n_out + tile * rows);
-        } else {
-            for (int a = 0; a < p.mt; ++a) tma_prefetch_2d(&tmA, kc, (tile * p.mt + a) * kBlockM);
-        }
-    };
     const int npre = min(p.stages, nkb);
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -205,7 +185,6 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
             mbar_expect_tx(full_bar(i), tx);
             load_a(base + (uint32_t)i * stage_bytes, full_bar(i), (kb0 + i) * kBlockK);
         }
-        for (int i = 0; i < p.pf_ahead; ++i) prefetch_a(npre + i);
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBh) : "memory");
         if (p.use_lo) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmBl) : "memory");
     }
@@ -240,7 +219,6 @@ __global__ void __launch_bounds__(320) gemm_tc_kernel(const __grid_constant__ CU
                 load_a(sa, full_bar(s), kc);
                 tma_load_2d(sa + a_bytes, &tmBh, full_bar(s), kc, 0);
                 if (p.use_lo) tma_load_2d(sa + a_bytes + b_bytes, &tmBl, full_bar(s), kc, 0);
-                if (p.pf_ahead) prefetch_a(i + p.pf_ahead);
             }
             // This lane does not reach the CTA's final barrier before every copy it issued has landed (the last
             // use of each stage; earlier uses were consumed before their stage was refilled).  It does so
