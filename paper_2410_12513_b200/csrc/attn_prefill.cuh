@@ -42,6 +42,8 @@ __global__ void __launch_bounds__(160, 2) attn_group_mma(const __grid_constant__
     constexpr int kKSteps = HD / 16, kNTiles = HD / 8;
     constexpr int GR = 2 * G;  // fragment rows of a warp: two tokens x G query heads
     static_assert(GR <= 8, "two tokens' query heads are the 8 hi rows of the A fragment");
+    static_assert((4 * GR * HD + 8 * GR) * 4 <= kStageBytes && 2 * 4 * GR * 64 * 4 <= kStageBytes,
+                  "the epilogue's scratch must fit the one stage a group is sure to hold");
 
     pdl_trigger();
     if (m_dev) m = min(m, __ldg(m_dev));
@@ -236,11 +238,14 @@ __global__ void __launch_bounds__(160, 2) attn_group_mma(const __grid_constant__
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar((tile0 + j) % kStages)) : "memory");
     };
 
-    // ---- each warp's rows are complete for this chunk: hand them over through shared memory (the ring is free)
+    // ---- each warp's rows are complete for this chunk: hand them over through shared memory
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
     bar_consumers();
-    float* o_s = reinterpret_cast<float*>(base_ptr);       // [4][GR][HD]
+    // Scratch = the stage of this group's LAST tile: the group holds it until release_last_stages, whereas any other
+    // stage may already be receiving the next group's tiles.  A stage (2 x HD x 128 B) holds the 4 x GR x HD floats
+    // and, later, the 2 x 32 x 64 merge weights.
+    float* o_s = reinterpret_cast<float*>(base_ptr + (size_t)((tile0 + n_tiles - 1) % kStages) * kStageBytes);  // [4][GR][HD]
     float* m_s = o_s + 4 * GR * HD;                         // [4][GR]
     float* l_s = m_s + 4 * GR;                              // [4][GR]
     if (g < GR) {
@@ -296,7 +301,7 @@ __global__ void __launch_bounds__(160, 2) attn_group_mma(const __grid_constant__
         continue;
     }
     __threadfence();
-    float* w_s = o_s;  // [kRows][64] weights, then [kRows][64] sums: 16 KB, the ring is free
+    float* w_s = o_s;  // [kRows][64] weights, then [kRows][64] sums: 16 KB, inside the same held stage
     for (int e = threadIdx.x; e < kRows * n_chunks; e += kConsumers) {
         const int r = e / n_chunks, sidx = e - r * n_chunks;
         float2 ml = make_float2(-INFINITY, 0.f);

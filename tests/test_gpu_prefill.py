@@ -152,6 +152,17 @@ def test_prefill_bf16_groups_of_eight(rows, chunk_tokens):
                   {"prefill_rows": rows, "attn_chunk": chunk_tokens})
 
 
+@pytest.mark.parametrize("hd", [64, 128])
+def test_prefill_bf16_many_tiny_prompts(hd):
+    """Dozens of prompts of one to five tokens side by side: almost every window of eight rows holds several group
+    leaders, which one attention CTA serves one after the other while its producer already fetches the next group's
+    tiles; a few longer prompts in between (several tiles, several token chunks)."""
+    shape = fi.ModelShape(2, 256, 8, 2, hd, 512, 2048, 500000.0)
+    lens = [1, 2, 3, 1, 1, 2, 5, 1, 4, 1, 150, 2, 1, 3, 1, 1, 70, 2, 2, 1, 5, 1, 1, 3, 9, 1, 2, 1, 1, 4] * 2
+    _prefill_case(shape, True, lens, 256, 1, 9, 1, 0.6, 2e-2, {"attn_chunk": 64})
+    _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2)
+
+
 def test_prefill_bf16_general_kernels_by_option():
     _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"attn_simple": 1, "max_gemv_rows": 1024})
 
