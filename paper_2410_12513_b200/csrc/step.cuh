@@ -198,9 +198,9 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
     if ((int)blockIdx.y >= m) return;
     const int i = blockIdx.y, head = blockIdx.x * blockDim.y + threadIdx.y, d = threadIdx.x, b = idx[i];
     if (head >= Hq + 2 * Hkv) return;
-    if (rowinfo && head == 0 && d == 0) {  // what attention needs to know about this row, in one 16-byte word
+    if (rowinfo && head == 0 && d < 32) {  // what attention needs to know about this row, in one 16-byte word
         long long y = (long long)slab_off[b];
-        if (pair) {
+        if (pair == 1 && d == 0) {
             // Prompt processing: rows i0, i0+1 that are consecutive tokens of one slab (the first at an even
             // position, both with room) share attention work items: bit 61 marks the first, bit 60 the second.
             auto is_pair = [&](int i0) {
@@ -210,30 +210,27 @@ __global__ void __launch_bounds__(512) rope_append(const float* qkv, const int32
                 return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == t0 + 1 &&
                        t0 + 1 < min(slab_cap[b1], cap_max) && !(t0 & 1);
             };
-            if (pair == 1) {
-                if (is_pair(i - 1)) y |= 1ll << 60;
-                else if (is_pair(i)) y |= 1ll << 61;
-            } else {
-                // Groups (attn_group_mma): up to eight consecutive tokens of one slab inside one block of eight
-                // positions.  A row leads a group unless it continues its predecessor's (again a local rule): bit 60
-                // = served by the leader; a leader carries its member count - 1 in bits 56..59.
-                auto consec = [&](int a) {  // rows a, a+1: consecutive tokens of one slab, the second with room
-                    if (a < 0 || a + 1 >= m) return false;
-                    const int b0 = idx[a], b1 = idx[a + 1];
-                    return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == len_l[b0] + 1 &&
-                           len_l[b1] < min(slab_cap[b1], cap_max);
-                };
-                const int p = len_l[b];
-                if (consec(i - 1) && (p & 7) != 0) {
-                    y |= 1ll << 60;
-                } else {
-                    int n = 1;
-                    while (n < 8 && ((p + n) & 7) != 0 && consec(i + n - 1)) ++n;
-                    y |= (long long)(n - 1) << 56;
-                }
-            }
+            if (is_pair(i - 1)) y |= 1ll << 60;
+            else if (is_pair(i)) y |= 1ll << 61;
+        } else if (pair == 2) {
+            // Groups (attn_group_mma): up to eight consecutive tokens of one slab inside one block of eight
+            // positions.  A row leads a group unless it continues its predecessor's (again a local rule): bit 60
+            // = served by the leader; a leader carries its member count - 1 in bits 56..59.  Lane d of the first
+            // warp looks at rows i+d-1, i+d (the eight pairs are independent, so they are looked at side by side).
+            auto consec = [&](int a) {  // rows a, a+1: consecutive tokens of one slab, the second with room
+                if (a < 0 || a + 1 >= m) return false;
+                const int b0 = idx[a], b1 = idx[a + 1];
+                return slab_off[b0] == slab_off[b1] && slab_cap[b0] == slab_cap[b1] && len_l[b1] == len_l[b0] + 1 &&
+                       len_l[b1] < min(slab_cap[b1], cap_max);
+            };
+            const int p = len_l[b];
+            const bool link = d < 8 && consec(i + d - 1) && ((p + d) & 7) != 0;  // row i+d continues row i+d-1's group
+            const unsigned links = __ballot_sync(__activemask(), link);
+            if (links & 1u) y |= 1ll << 60;
+            else y |= (long long)(__ffs(~((links >> 1) & 0x7fu)) - 1) << 56;  // members after the leader: leading links
         }
-        rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, min(slab_cap[b], cap_max)) | ((long long)b << 32), y);
+        if (d == 0)
+            rowinfo[i] = make_longlong2((long long)min(len_l[b] + 1, min(slab_cap[b], cap_max)) | ((long long)b << 32), y);
     }
     const int half = hd >> 1;
     const int qd = Hq * hd, kvd = Hkv * hd;
