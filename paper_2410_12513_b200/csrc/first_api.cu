@@ -10,6 +10,7 @@
 
 #include "attn_mma.cuh"
 #include "attn_prefill.cuh"
+#include "attn_prefill_tc.cuh"
 #include "attn_simple.cuh"
 #include "common.cuh"
 #include "first.h"
@@ -109,6 +110,7 @@ struct first_ctx {
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
     int prefill_group = 1; // prompt chunks: up to eight consecutive tokens share one (takes precedence over pairs)
+    int prefill_tc = 0;    // prompt chunks: attention on the tcgen05 tensor cores, blocks of 128/G tokens (takes precedence over groups)
     int prefill_rows = 0;  // rows per prompt chunk (0: 256)
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted
@@ -617,6 +619,8 @@ int attn_mma_set_attr() {
     constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     CU_TRY(cudaFuncSetAttribute(attn::attn_split_mma<HD, G, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024));
+    CU_TRY(cudaFuncSetAttribute(attn::attn_prefill_tc<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                attn::PrefillTc<HD, G>::kSmem));
     if constexpr (2 * G <= 8)  // the group form used on prompt chunks
         CU_TRY(cudaFuncSetAttribute(attn::attn_group_mma<HD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     if constexpr (2 * G <= 8)  // the two-rows-per-work-item form used on prompt chunks
@@ -650,6 +654,13 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
         // many rows: whole rows already fill the CTA slots several times over, and an unsplit row needs no merge
         if (m * d.n_kv_heads >= 3 * c->n_sm && d.max_tokens_per_seq <= 2048) C = d.max_tokens_per_seq;
     }
+    if (pair == 3 && c->attn_chunk <= 0) {
+        // blocks of 128/G tokens: (m * G / 128) * Hkv work items per token chunk, one CTA per SM -- cut the token
+        // axis so that the longest rows' items just about fill the SMs
+        const double items = std::max(1.0, (double)m * c->group / 128.0) * d.n_kv_heads;
+        C = std::max(256, (int)(d.max_tokens_per_seq * std::min(1.0, items / c->n_sm)));
+    }
+    if (pair == 3) C = std::max(C, (d.max_tokens_per_seq + 31) / 32);  // (its merge keeps 32 chunks' weights per row)
     C = std::max(C, (d.max_tokens_per_seq + c->max_splits - 1) / c->max_splits);
     C = (C + attn::kTile - 1) / attn::kTile * attn::kTile;
     const int S = (d.max_tokens_per_seq + C - 1) / C;
@@ -657,6 +668,17 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
     int rc;
     if ((rc = kv_map_for(c, kc, kv->cap_total, &tk)) || (rc = kv_map_for(c, vc, kv->cap_total, &tv))) return rc;
     dim3 grid(S, d.n_kv_heads, m);
+#define FIRST_ATTN_TC(HD, G)                                                                                     \
+    if (pair == 3 && d.head_dim == HD && c->group == G) {                                                        \
+        constexpr int TQ = attn::PrefillTc<HD, G>::TQ;                                                           \
+        return launch_k(c, st, kClsAttn, attn::attn_prefill_tc<HD, G>, dim3(grid.y, (m + TQ - 1) / TQ + 1, grid.x), \
+                        dim3(attn::kTcThreads), attn::PrefillTc<HD, G>::kSmem, *tk, *tv, c->q, kv->cap_total,    \
+                        c->rowinfo, m, m_dev, d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out, out_hi,     \
+                        out_lo, c->flags);                                                                       \
+    }
+    FIRST_ATTN_TC(128, 1) FIRST_ATTN_TC(128, 2) FIRST_ATTN_TC(128, 3) FIRST_ATTN_TC(128, 4) FIRST_ATTN_TC(128, 8)
+    FIRST_ATTN_TC(64, 1) FIRST_ATTN_TC(64, 2) FIRST_ATTN_TC(64, 3) FIRST_ATTN_TC(64, 4) FIRST_ATTN_TC(64, 8)
+#undef FIRST_ATTN_TC
 #define FIRST_ATTN_GROUP(HD, G)                                                                                  \
     if (pair == 2 && d.head_dim == HD && c->group == G) {                                                        \
         constexpr int smem = attn::kStages * 2 * (HD / 64) * attn::kTile * 128 + 1024;                           \
@@ -732,7 +754,11 @@ int decode_step_impl(first_ctx* c, const int32_t* tokens, const first_kv_cache* 
     // prompt chunks: consecutive rows are consecutive tokens of a sequence and may share attention work items
     const bool route_here = ph && ph->router_w;
     // (0 = each row its own work items, 1 = pairs of consecutive tokens, 2 = groups of up to eight)
-    const int pair_rows = (ph && mma_attn && !fuse_rope && 2 * c->group <= 8) ? (c->prefill_group ? 2 : c->prefill_pair ? 1 : 0) : 0;
+    // (3 = blocks of 128/G tokens on the tcgen05 tensor cores)
+    const bool tc_blocks = ph && mma_attn && !fuse_rope && c->prefill_tc && B <= attn::kTcMaxRows &&
+                           (c->group == 1 || c->group == 2 || c->group == 3 || c->group == 4 || c->group == 8);
+    const int pair_rows = tc_blocks ? 3
+                          : (ph && mma_attn && !fuse_rope && 2 * c->group <= 8) ? (c->prefill_group ? 2 : c->prefill_pair ? 1 : 0) : 0;
 
     for (int l = 0; l < L; ++l) {
         if (layer_inputs) {
@@ -1342,6 +1368,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "fuse_rope")) c->fuse_rope = value != 0;
     else if (!std::strcmp(name, "prefill_pair")) c->prefill_pair = value != 0;
     else if (!std::strcmp(name, "prefill_group")) c->prefill_group = value != 0;
+    else if (!std::strcmp(name, "prefill_tc")) c->prefill_tc = value != 0;
     else if (!std::strcmp(name, "prefill_rows")) c->prefill_rows = value > 0 ? (int)value : 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;

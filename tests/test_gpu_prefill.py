@@ -163,6 +163,32 @@ def test_prefill_bf16_many_tiny_prompts(hd):
     _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2)
 
 
+@pytest.mark.parametrize("rows,chunk_tokens", [(20, 64), (256, 64), (37, 128), (256, 1024)])
+def test_prefill_bf16_tensor_core_blocks(rows, chunk_tokens):
+    """Attention of prompt chunks on the tcgen05 tensor cores (option `prefill_tc`): blocks of 128/G consecutive
+    tokens per work item, at chunk heights that cut blocks at odd places, with prompts of 1 .. 300 tokens (blocks of
+    every size, sequences that start in the middle of a chunk, several tiles and several token chunks per block)."""
+    _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 7, 8, 9, 300, 16], rows, 2, 8, 1, 0.6, 2e-2,
+                  {"prefill_rows": rows, "attn_chunk": chunk_tokens, "prefill_tc": 1})
+
+
+@pytest.mark.parametrize("hq,hkv,hd", [(4, 4, 64), (4, 2, 128), (6, 2, 64), (8, 1, 64), (8, 2, 128), (6, 2, 128)])
+def test_prefill_bf16_tensor_core_blocks_head_groupings(hq, hkv, hd):
+    """1, 2, 3, 4 and 8 query heads per KV head at both head sizes: blocks of 128, 64, 42, 32 and 16 tokens."""
+    shape = fi.ModelShape(2, hq * hd, hq, hkv, hd, 512, 1024, 500000.0)
+    _prefill_case(shape, True, [70, 3, 131, 260], 256, 2, 8, 0, 0.6, 2e-2, {"prefill_tc": 1})
+
+
+@pytest.mark.parametrize("hd", [64, 128])
+def test_prefill_bf16_tensor_core_blocks_many_tiny_prompts(hd):
+    """Dozens of prompts of one to five tokens side by side: a window of 32 rows holds many block starts, which one
+    CTA serves one after the other (ring stages, buffer parities and barrier phases run on from block to block)."""
+    shape = fi.ModelShape(2, 256, 8, 2, hd, 512, 2048, 500000.0)
+    lens = [1, 2, 3, 1, 1, 2, 5, 1, 4, 1, 150, 2, 1, 3, 1, 1, 70, 2, 2, 1, 5, 1, 1, 3, 9, 1, 2, 1, 1, 4] * 2
+    _prefill_case(shape, True, lens, 256, 1, 9, 1, 0.6, 2e-2, {"attn_chunk": 64, "prefill_tc": 1})
+    _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2, {"prefill_tc": 1})
+
+
 def test_prefill_bf16_general_kernels_by_option():
     _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"attn_simple": 1, "max_gemv_rows": 1024})
 
