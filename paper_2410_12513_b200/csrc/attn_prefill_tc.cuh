@@ -8,25 +8,32 @@
 //   S  = (Q_hi + Q_lo) K^T      tcgen05.mma, Q and K K-major in 128-byte-swizzled shared memory, S in tensor memory
 //   P  = exp(S - max)           four warps, one row per thread (tcgen05.ld), causal mask, online softmax; the weights
 //                               go back into the columns S came from as packed bfloat16 pairs (tcgen05.st)
-//   PV = (P_hi + P_lo) V        tcgen05.mma with A = P read from tensor memory, V as the TMA left it ([token][dim]:
-//                               an MN-major B operand), PV in tensor memory, added to the thread's output row
+//   O += (P_hi + P_lo) V        tcgen05.mma with A = P read from tensor memory, V as the TMA left it ([token][dim]:
+//                               an MN-major B operand); O stays in tensor memory over all tiles of the block
+// The weights are taken relative to a reference maximum m_ref that follows the running maximum lazily: only when
+// a tile's maximum exceeds m_ref by more than 8 (base-2 exponent) is m_ref moved and O (and the running sum)
+// scaled down; in between weights may be as large as 2^8, which float32 sums and the bfloat16 hi/lo split carry
+// without loss.  O / sum at the end does not depend on which reference was used.
 // Operands fetched from shared memory cost the tensor pipe time (measured: about 64 bytes per clock, so a
 // 128 x 64 x 16 MMA with both operands there takes 90 clocks instead of 32): hence tiles of 128 tokens for S and P
 // kept in tensor memory for PV.  Precision is that of the other attention kernels: q and the softmax weights are
-// split into bfloat16 hi + lo against the stored bfloat16 keys and values, float32 accumulation.  S/P and PV are
+// split into bfloat16 hi + lo against the stored bfloat16 keys and values, float32 accumulation.  S/P is
 // double-buffered in tensor memory, so the tensor pipe computes S of tile j+1 while the softmax warps work on tile j.
 // The token axis is cut into chunks per CTA; the CTA that finishes a (block, kv head) last merges the chunks
 // (atomic ticket), as in the decode kernel.
 //
-// Roles (192 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1 owns the tensor memory),
-// warps 2..5 = softmax and epilogue (tensor-memory lane quadrant = warp % 4).  Every wait is bounded.
+// Roles (320 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1 owns the tensor memory),
+// warps 2..5 and 6..9 = two softmax warpgroups (tensor-memory lane quadrant = warp % 4): a row of the tile belongs
+// to one thread of each, the first takes tokens 0..63 of every tile and the first half of the output row, the second
+// the rest; they exchange their row maxima through shared memory once per tile (one warp per scheduler alone spends
+// its time waiting for its own exp2 and tensor-memory results).  Every wait is bounded.
 #pragma once
 #include "attn_mma.cuh"
 
 namespace first {
 namespace attn {
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
 constexpr int kTcMaxRows = 256;  // rows of a launch (a prompt chunk)
 
 // MN-major operand in 128-byte-swizzled rows (row = one K index, 64 MN elements wide): 8-row groups 1024 bytes
@@ -53,6 +60,10 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
         ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
           "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // D[tmem] (+)= A[tmem] * B[smem]: A's row i sits in lane i, two consecutive K elements per 32-bit column
 __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t acc) {
@@ -75,6 +86,7 @@ __device__ __forceinline__ void split2_trunc(float x, float y, uint32_t& hi, uin
     const float xl = x - __uint_as_float(xb & 0xffff0000u), yl = y - __uint_as_float(yb & 0xffff0000u);
     lo = __byte_perm(__float_as_uint(xl), __float_as_uint(yl), 0x7632);
 }
+__device__ __forceinline__ void bar_softmax() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -89,10 +101,10 @@ struct PrefillTc {
     static constexpr int kTileBytes = kHalves * kHalfBytes;  // a K tile or a V tile
     static constexpr int kQBytes = 2 * kTileBytes;         // hi halves, then lo halves
     static constexpr int kSmem = kQBytes + 4 * kTileBytes + 1024;  // Q, two K tiles, two V tiles
-    static constexpr int kTmemCols = HD == 128 ? 512 : 512;  // S/P: 2 x 128 columns, PV: 2 x HD columns (power of two)
+    static constexpr int kTmemCols = 512;  // S/P: 2 x 128 columns, O: HD columns (power of two)
 };
 
-// grid (Hkv, Z, S_max), 192 threads, at most 256 rows: CTA (h, z, c) serves the z-th, (z+Z)-th, ... block of the
+// grid (Hkv, Z, S_max), 320 threads, at most 256 rows: CTA (h, z, c) serves the z-th, (z+Z)-th, ... block of the
 // launch (so with Z >= the number of blocks, one each; the host takes Z = ceil(m / TQ) + 1, which covers a chunk that
 // lies inside one sequence) for KV head h and token chunk c; chunks are the slowest grid dimension, so the CTAs
 // of chunks that few rows reach come last.  A block starts at row i when i is the launch's first row, when row i is
@@ -101,7 +113,7 @@ struct PrefillTc {
 // q: [m][Hq][HD] float32, rotated and pre-scaled.  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64 x 64.  Scratch and
 // outputs as in attn_split_mma (o_part [m][Hq][S_max][HD], ml_part [m][Hq][S_max], ticket [m][Hkv]).
 template <int HD, int G>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 1)  // (ten warps: three share a scheduler's registers, 168 each)
 attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const float* q,
                 int64_t cap_total, const longlong2* rowinfo, int m, const int32_t* __restrict__ m_dev, int Hq, int C,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, uint32_t* __restrict__ ticket,
@@ -112,7 +124,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     constexpr int TQ = P::TQ, kTok = P::kTok, kHalves = P::kHalves, kBox = P::kBox, kHalfBytes = P::kHalfBytes;
     constexpr int kTileBytes = P::kTileBytes;
     constexpr int kRows = TQ * G;        // MMA rows that can carry a query head (the rest stay zero)
-    constexpr int kPvCol0 = 2 * kTok;    // tensor-memory column of the first PV buffer
+    constexpr int kOCol0 = 2 * kTok;     // tensor-memory column of the output accumulator
 
     pdl_trigger();
     if (m_dev) m = min(m, __ldg(m_dev));
@@ -122,6 +134,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     __shared__ int abort_s;
     __shared__ int last_s;
     __shared__ uint32_t lead_s[kTcMaxRows / 32];  // bit i = row i starts a block
+    __shared__ float xch_s[2][2][128];            // [tile parity][warpgroup][row]: row maxima (sums at the end)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.x, c = blockIdx.z, Hkv = gridDim.x, S_max = gridDim.z;
     const int Ce = (C + kTok - 1) / kTok * kTok;  // chunk length in whole tiles
@@ -191,10 +204,10 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             tc::mbar_init(v_full(b), 1);
             tc::mbar_init(v_empty(b), 1);
             tc::mbar_init(s_full(b), 1);
-            tc::mbar_init(p_full(b), 4);
+            tc::mbar_init(p_full(b), 8);
             tc::mbar_init(pv_full(b), 1);
         }
-        tc::mbar_init(q_full, 4);
+        tc::mbar_init(q_full, 8);
         tc::mbar_init(done_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -295,13 +308,13 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t dv = dv0 + (uint64_t)((uint32_t)b * (kTileBytes >> 4));
                     const uint32_t ta = tmem + (uint32_t)(b * kTok);   // P where S was: per 64 tokens 32 columns hi, 32 lo
-                    const uint32_t td = tmem + (uint32_t)(kPvCol0 + b * HD);
+                    const uint32_t td = tmem + (uint32_t)kOCol0;
 #pragma unroll
                     for (int part = 0; part < 2; ++part)  // p_hi, then p_lo
 #pragma unroll
                         for (int k = 0; k < kTok / 16; ++k)
                             umma_bf16_ts(td, ta + (uint32_t)((k >> 2) * 64 + part * 32 + (k & 3) * 8), dv + (uint64_t)((k * 2048) >> 4),
-                                         idesc_pv, (part | k) ? 1u : 0u);
+                                         idesc_pv, (j | part | k) ? 1u : 0u);  // the block's first MMA starts O afresh
                     tc::umma_commit(v_empty(b));  // the V tile is free once these MMAs have read it
                     tc::umma_commit(pv_full(b));
                 }
@@ -309,17 +322,19 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             continue;
         }
 
-        // ---------------- softmax warps: thread = one MMA row
+        // ---------------- softmax warpgroups: a row of the tile = one thread of each
+        const int st = (int)threadIdx.x - 64, wg = st >> 7;   // wg: which half of the tile's tokens and of the output row
         const int quad = warp & 3, r = quad * 32 + lane;
         const int tok = r / G, gq = r - tok * G;
         const bool live = r < kRows && tok < n;
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+        constexpr int HH = HD / 2;  // output columns of a thread
         {   // Q of this block: float32 -> bfloat16 hi/lo, K-major swizzled rows (the previous block's MMAs are done:
-            // its last PV was waited for).  Warp w converts rows 32w .. 32w+31, a row (or two) per pass.
+            // its last PV was waited for).  Warp w converts rows 16w .. 16w+15.
             const int sw = warp - 2;
 #pragma unroll 8
-            for (int e = lane; e < 32 * HD / 4; e += 32) {
-                const int rq = sw * 32 + e / (HD / 4), d4 = (e % (HD / 4)) * 4;
+            for (int e = lane; e < 16 * HD / 4; e += 32) {
+                const int rq = sw * 16 + e / (HD / 4), d4 = (e % (HD / 4)) * 4;
                 const int tq = rq / G, gg = rq - tq * G;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (rq < kRows && tq < n)
@@ -337,175 +352,183 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(q_full);
         }
-        float o[HD];
-#pragma unroll
-        for (int d = 0; d < HD; ++d) o[d] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f, alpha = 1.f;
+        float m_ref = -INFINITY, l_run = 0.f;
+        // A failed wait makes `ok` false for good, for the whole warp (the tensor-memory instructions below want the
+        // warp together); the warp still goes through every barrier of the loop (its partner and the other warps
+        // wait there), only the work is skipped.
         bool ok = true;
         // this row sees tokens t < see of this chunk's range; a row without a query head (all-zero q) is never
         // written out and takes the unmasked path
         const int see = live ? min(T1 + tok, t_end) : 0x7fffffff;
         constexpr float kLog2e = 1.4426950408889634f;
-        auto add_pv = [&](int jj, float scale) {  // o = (o + PV of tile jj) * scale
-            if (!tc::mbar_wait(pv_full(jj & 1), (uint32_t)(jj >> 1) & 1u, &abort_s, flags)) return false;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t ta = lane_addr + (uint32_t)(kPvCol0 + (jj & 1) * HD);
-            uint32_t v[2][32];
-            tmem_ld16_nowait(ta, v[0]);
-            tmem_ld16_nowait(ta + 16u, v[0] + 16);
-#pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 32) {
-                const int cur = (c0 >> 5) & 1;
-                tmem_ld_wait();
-                if (c0 + 32 < HD) {  // the next 32 columns travel while these are added
-                    tmem_ld16_nowait(ta + (uint32_t)(c0 + 32), v[cur ^ 1]);
-                    tmem_ld16_nowait(ta + (uint32_t)(c0 + 48), v[cur ^ 1] + 16);
-                }
-                if (scale == 1.f) {  // the running maximum did not move: nothing to rescale
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) o[c0 + k] += __uint_as_float(v[cur][k]);
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) o[c0 + k] = (o[c0 + k] + __uint_as_float(v[cur][k])) * scale;
-                }
-            }
-            return true;
-        };
+        constexpr float kSlack = 8.f / kLog2e;  // m_ref moves only when a tile's maximum is this far above it
+        const uint32_t o_addr = lane_addr + (uint32_t)(kOCol0 + wg * HH);  // this thread's half of the output row
         for (int j = 0; j < n_tiles; ++j) {
             const int jj = tile0 + j, b = jj & 1;
-            if (!tc::mbar_wait(s_full(b), (uint32_t)(jj >> 1) & 1u, &abort_s, flags)) { ok = false; break; }
+            ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(s_full(b), (uint32_t)(jj >> 1) & 1u, &abort_s, flags));
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t s_addr = lane_addr + (uint32_t)(b * kTok);
+            const uint32_t s_addr = lane_addr + (uint32_t)(b * kTok + wg * 64);  // this thread's 64 columns
             const int t0 = t_begin + j * kTok;
-            const int lim = see - t0;          // columns of this tile the row sees
-            const bool whole = lim >= kTok;    // every column visible: the usual case away from the diagonal
-            // pass 1: the row's maximum over the tile (64 columns at a time)
+            const int lim = see - t0 - wg * 64;  // columns of this thread's half the row sees
+            const bool whole = lim >= 64;        // every column visible: the usual case away from the diagonal
+            uint32_t sv[64];
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (ok) {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t sv[64];
-#pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16_nowait(s_addr + (uint32_t)(hh * 64 + c0), sv + c0);
+                for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16_nowait(s_addr + (uint32_t)c0, sv + c0);
                 tmem_ld_wait();
                 if (whole) {
 #pragma unroll
                     for (int k = 0; k < 64; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(sv[k]));
                 } else {
 #pragma unroll
-                    for (int k = 0; k < 64; ++k)
-                        if (hh * 64 + k < lim) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(sv[k]));
+                    for (int k = 0; k < 64; ++k) {
+                        if (k >= lim) sv[k] = 0xff800000u;  // -inf: weight 0
+                        mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(sv[k]));
+                    }
                 }
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            const float m_new = fmaxf(m_run, mx);
-            alpha = (m_new == -INFINITY) ? 1.f : (m_run == -INFINITY ? 0.f : ex2_approx((m_run - m_new) * kLog2e));
-            m_run = m_new;
-            const float mb = (m_new == -INFINITY) ? 0.f : m_new * kLog2e;  // (then no column is visible: weights 0)
-            // pass 2: weights, their sum, and P back into the columns S came from: per 64 tokens 32 columns of
-            // bfloat16 pairs (hi), then 32 (lo) -- exactly the 64 columns whose S values are in registers by then
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            xch_s[b][wg][r] = mx;
+            bar_softmax();
+            mx = fmaxf(mx, xch_s[b][wg ^ 1][r]);  // (written again two tiles on, a barrier later)
+            float alpha = 1.f;
+            if (m_ref == -INFINITY) {
+                m_ref = mx;  // first visible column (or still none): nothing accumulated yet
+            } else if (mx > m_ref + kSlack) {
+                alpha = ex2_approx((m_ref - mx) * kLog2e);
+                m_ref = mx;
+                l_run *= alpha;
+            }
+            const float mb = (m_ref == -INFINITY) ? 0.f : m_ref * kLog2e;  // (then no column is visible: weights 0)
+            // weights, their sum, and P back into the columns S came from: 32 columns of bfloat16 pairs (hi), then
+            // 32 (lo) -- exactly this thread's 64 columns, whose S values are in its registers
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            if (ok) {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t sv[64];
+                for (int qd = 0; qd < 4; ++qd) {  // 16 tokens -> 8 columns hi, 8 columns lo
+                    uint32_t phi[8], plo[8];
 #pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16_nowait(s_addr + (uint32_t)(hh * 64 + c0), sv + c0);
-                tmem_ld_wait();
-#pragma unroll
-                for (int qd = 0; qd < 2; ++qd) {  // 32 tokens -> 16 columns hi, 16 columns lo
-                    uint32_t phi[16], plo[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const int col = qd * 32 + 2 * k;
-                        float p0 = ex2_approx(fmaf(__uint_as_float(sv[col]), kLog2e, -mb));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(sv[col + 1]), kLog2e, -mb));
-                        if (!whole) {
-                            if (hh * 64 + col >= lim) p0 = 0.f;
-                            if (hh * 64 + col + 1 >= lim) p1 = 0.f;
-                        }
+                    for (int k = 0; k < 8; ++k) {
+                        const int col = qd * 16 + 2 * k;
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(sv[col]), kLog2e, -mb));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(sv[col + 1]), kLog2e, -mb));
                         sum4[k & 3] += p0 + p1;
                         split2_trunc(p0, p1, phi[k], plo[k]);
                     }
-                    tmem_st16(s_addr + (uint32_t)(hh * 64 + qd * 16), phi);
-                    tmem_st16(s_addr + (uint32_t)(hh * 64 + 32 + qd * 16), plo);
+                    tmem_st8(s_addr + (uint32_t)(qd * 8), phi);
+                    tmem_st8(s_addr + (uint32_t)(32 + qd * 8), plo);
                 }
             }
-            l_run = l_run * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+            l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             if (t0 + kTok > T) {
                 // rows past the sequence's end hold someone else's bytes: zero them in V so that 0 * garbage stays 0
                 const int valid = T - t0;
-                if (!tc::mbar_wait(v_full(b), (uint32_t)(jj >> 1) & 1u, &abort_s, flags)) { ok = false; break; }
+                ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(v_full(b), (uint32_t)(jj >> 1) & 1u, &abort_s, flags));
                 uint8_t* vptr = base_ptr + P::kQBytes + 2 * kTileBytes + (size_t)b * kTileBytes;
-                for (int e = (int)threadIdx.x - 64; e < (kTok - valid) * kHalves * 8; e += 128) {
-                    const int row = valid + e / (kHalves * 8), cc = e % (kHalves * 8);
-                    *reinterpret_cast<uint4*>(vptr + (cc >> 3) * kHalfBytes + row * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
-                }
+                if (ok)
+                    for (int e = st; e < (kTok - valid) * kHalves * 8; e += 256) {
+                        const int row = valid + e / (kHalves * 8), cc = e % (kHalves * 8);
+                        *reinterpret_cast<uint4*>(vptr + (cc >> 3) * kHalfBytes + row * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
                 fence_async_smem();
+            }
+            // O holds tiles 0 .. j-1 once PV of tile j-1 is done.  Waited for every tile (the barrier's phases are taken
+            // in order) but only here, after the weights: by now that PV is over unless the tensor pipe is the slower side.
+            if (j > 0) ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(pv_full((jj - 1) & 1), (uint32_t)((jj - 1) >> 1) & 1u, &abort_s, flags));
+            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f) && ok) {
+                // some row of this warp moved its reference: scale this warp's rows of O (1 for the others)
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int c0 = 0; c0 < HH; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld16_nowait(o_addr + (uint32_t)c0, v);
+                    tmem_ld16_nowait(o_addr + (uint32_t)(c0 + 16), v + 16);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
+                    tmem_st16(o_addr + (uint32_t)c0, v);
+                    tmem_st16(o_addr + (uint32_t)(c0 + 16), v + 16);
+                }
             }
             tmem_st_wait();
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(b));
-            if (j > 0 && !add_pv(jj - 1, alpha)) { ok = false; break; }
+            if (lane == 0 && ok) mbar_arrive(p_full(b));
         }
-        if (ok) ok = add_pv(tile0 + n_tiles - 1, 1.f);
+        // the block's output: O is complete once the last PV is
+        ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(pv_full((tile0 + n_tiles - 1) & 1), (uint32_t)((tile0 + n_tiles - 1) >> 1) & 1u, &abort_s, flags));
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float o[HH];
+        if (ok) {
+#pragma unroll
+            for (int c0 = 0; c0 < HH; c0 += 16) tmem_ld16_nowait(o_addr + (uint32_t)c0, reinterpret_cast<uint32_t*>(o) + c0);
+            tmem_ld_wait();
+        }
+        // the row's sum: both halves
+        xch_s[0][wg][r] = l_run;
+        bar_softmax();
+        const float l_tot = l_run + xch_s[0][wg ^ 1][r];
+        bar_softmax();  // (xch_s is written again by the next block's first tile)
         ok = ok && !abort_s;
-        // ---------------- epilogue: the thread holds its row's unnormalised output, maximum and sum
+        // ---------------- epilogue: the thread holds its half of the row's unnormalised output, the maximum and the sum
         const size_t hq = ((size_t)(i0 + tok) * Hq + (size_t)h * G + gq);
-        auto emit_row = [&](float scale) {
-            if (out) {
+        if (n_chunks == 1) {
+            if (ok && live) {
+                const float scale = 1.f / l_tot;
+                const size_t o0 = hq * HD + (size_t)wg * HH;
+                if (out) {
 #pragma unroll
-                for (int d = 0; d < HD; d += 4)
-                    *reinterpret_cast<float4*>(out + hq * HD + d) =
-                        make_float4(o[d] * scale, o[d + 1] * scale, o[d + 2] * scale, o[d + 3] * scale);
-            }
-            if (out_hi) {
+                    for (int d = 0; d < HH; d += 4)
+                        *reinterpret_cast<float4*>(out + o0 + d) =
+                            make_float4(o[d] * scale, o[d + 1] * scale, o[d + 2] * scale, o[d + 3] * scale);
+                }
+                if (out_hi) {
 #pragma unroll
-                for (int d = 0; d < HD; d += 8) {
-                    uint4 hi, lo;
-                    split2(o[d] * scale, o[d + 1] * scale, hi.x, lo.x);
-                    split2(o[d + 2] * scale, o[d + 3] * scale, hi.y, lo.y);
-                    split2(o[d + 4] * scale, o[d + 5] * scale, hi.z, lo.z);
-                    split2(o[d + 6] * scale, o[d + 7] * scale, hi.w, lo.w);
-                    *reinterpret_cast<uint4*>(out_hi + hq * HD + d) = hi;
-                    *reinterpret_cast<uint4*>(out_lo + hq * HD + d) = lo;
+                    for (int d = 0; d < HH; d += 8) {
+                        uint4 hi, lo;
+                        split2(o[d] * scale, o[d + 1] * scale, hi.x, lo.x);
+                        split2(o[d + 2] * scale, o[d + 3] * scale, hi.y, lo.y);
+                        split2(o[d + 4] * scale, o[d + 5] * scale, hi.z, lo.z);
+                        split2(o[d + 6] * scale, o[d + 7] * scale, hi.w, lo.w);
+                        *reinterpret_cast<uint4*>(out_hi + o0 + d) = hi;
+                        *reinterpret_cast<uint4*>(out_lo + o0 + d) = lo;
+                    }
                 }
             }
-        };
-        if (n_chunks == 1) {
-            if (ok && live) emit_row(1.f / l_run);
             continue;
         }
         if (ok && live) {
 #pragma unroll
-            for (int d = 0; d < HD; d += 4)
-                *reinterpret_cast<float4*>(o_part + (hq * S_max + c) * HD + d) = make_float4(o[d], o[d + 1], o[d + 2], o[d + 3]);
-            ml_part[hq * S_max + c] = make_float2(m_run, l_run);
+            for (int d = 0; d < HH; d += 4)
+                *reinterpret_cast<float4*>(o_part + (hq * S_max + c) * HD + wg * HH + d) = make_float4(o[d], o[d + 1], o[d + 2], o[d + 3]);
+            if (wg == 0) ml_part[hq * S_max + c] = make_float2(m_ref, l_tot);
         }
         // ticket: the last chunk of this (block, kv head) to get here merges them all
         __threadfence();
-        bar_consumers();
+        bar_softmax();
         if (threadIdx.x == 64) {
             const uint32_t t = ok ? atomicAdd(&ticket[(size_t)i0 * Hkv + h], 1u) : 0u;
             last_s = ok && (t == (uint32_t)n_chunks - 1u);
             if (last_s) ticket[(size_t)i0 * Hkv + h] = 0u;
         }
-        bar_consumers();
+        bar_softmax();
         const bool last = last_s != 0;
-        bar_consumers();  // (last_s is written again by the next block)
+        bar_softmax();  // (last_s is written again by the next block)
         if (!last) continue;
         __threadfence();
-        // Merge, all 128 threads side by side (a thread per row would wait for one load after the other):
+        // Merge, all 256 threads side by side (a thread per row would wait for one load after the other):
         // (1) every chunk's (max, sum) into shared memory -- Q's memory is free, the block's MMAs are done --
-        // (2) one weight per (row, chunk), (3) weighted sums, four (eight) rows per pass with coalesced loads.
+        // (2) one weight per (row, chunk), (3) weighted sums, eight (sixteen) rows per pass with coalesced loads.
         {
-            const int rows_live = n * G, tid = (int)threadIdx.x - 64;
+            const int rows_live = n * G, tid = st;
             float2* w_s = reinterpret_cast<float2*>(base_ptr);  // [rows_live][n_chunks]
             auto hq_of = [&](int rw) { return (size_t)(i0 + rw / G) * Hq + (size_t)h * G + rw % G; };
-            for (int e = tid; e < rows_live * n_chunks; e += 128) {
+            for (int e = tid; e < rows_live * n_chunks; e += 256) {
                 const int rw = e / n_chunks, sidx = e - rw * n_chunks;
                 w_s[e] = __ldcg(&ml_part[hq_of(rw) * S_max + sidx]);
             }
-            bar_consumers();
+            bar_softmax();
             if (tid < rows_live) {
                 float2* wr = w_s + tid * n_chunks;
                 float M = -INFINITY, den = 0.f;
@@ -514,8 +537,8 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float inv = 1.f / den;
                 for (int sidx = 0; sidx < n_chunks; ++sidx) wr[sidx].x = __expf(wr[sidx].x - M) * inv;
             }
-            bar_consumers();
-            constexpr int LPR = HD / 4, RPP = 128 / LPR;  // lanes per row (a float4 each), rows per pass
+            bar_softmax();
+            constexpr int LPR = HD / 4, RPP = 256 / LPR;  // lanes per row (a float4 each), rows per pass
             const int d4 = (tid % LPR) * 4;
 #pragma unroll 2
             for (int rb = 0; rb < rows_live; rb += RPP) {
@@ -544,7 +567,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
             }
-            bar_consumers();  // (the next block's Q goes where the weights are)
+            bar_softmax();  // (the next block's Q goes where the weights are)
         }
     }
 

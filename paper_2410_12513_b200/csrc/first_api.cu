@@ -110,7 +110,7 @@ struct first_ctx {
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
     int prefill_group = 1; // prompt chunks: up to eight consecutive tokens share one (takes precedence over pairs)
-    int prefill_tc = 0;    // prompt chunks: attention on the tcgen05 tensor cores, blocks of 128/G tokens (takes precedence over groups)
+    int prefill_tc = 1;    // prompt chunks: attention on the tcgen05 tensor cores, blocks of 128/G tokens (takes precedence over groups)
     int prefill_rows = 0;  // rows per prompt chunk (0: 256)
     int tune_pair_rows = 1;
     int tc_smem_kb = 110;  // shared-memory budget per projection CTA when two CTAs per SM are wanted

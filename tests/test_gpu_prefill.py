@@ -134,22 +134,22 @@ def test_prefill_bf16_query_head_groupings(hq, hkv, hd):
 def test_prefill_bf16_pairing_off_by_option():
     """Every prompt token with attention work items of its own (neither groups of eight nor pairs)."""
     _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2,
-                  {"prefill_group": 0, "prefill_pair": 0, "prefill_rows": 20})
+                  {"prefill_tc": 0, "prefill_group": 0, "prefill_pair": 0, "prefill_rows": 20})
 
 
 def test_prefill_bf16_pairs_by_option():
-    """The pair form (two consecutive tokens per work item), which groups of eight replaced as the default."""
-    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"prefill_group": 0, "prefill_rows": 20})
-    _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 200], 256, 2, 7, 0, 0.6, 2e-2, {"prefill_group": 0})
+    """The pair form (two consecutive tokens per work item), which groups of eight replaced (option `prefill_tc` 0, `prefill_group` 0)."""
+    _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"prefill_tc": 0, "prefill_group": 0, "prefill_rows": 20})
+    _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 200], 256, 2, 7, 0, 0.6, 2e-2, {"prefill_tc": 0, "prefill_group": 0})
 
 
 @pytest.mark.parametrize("rows,chunk_tokens", [(20, 64), (256, 64), (37, 128), (256, 1024)])
 def test_prefill_bf16_groups_of_eight(rows, chunk_tokens):
-    """Groups of up to eight consecutive tokens per attention work item (the default), at chunk heights that cut
+    """Groups of up to eight consecutive tokens per attention work item (`prefill_tc` 0: the mma.sync form), at chunk heights that cut
     groups at odd places (20, 37 rows), with prompts of 1, 2, 7, 8, 9 tokens (groups of every size, sequences that
     start in the middle of a chunk) and prompts long enough for several token chunks per group (merged by ticket)."""
     _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 7, 8, 9, 300, 16], rows, 2, 8, 1, 0.6, 2e-2,
-                  {"prefill_rows": rows, "attn_chunk": chunk_tokens})
+                  {"prefill_tc": 0, "prefill_rows": rows, "attn_chunk": chunk_tokens})
 
 
 @pytest.mark.parametrize("hd", [64, 128])
@@ -159,13 +159,13 @@ def test_prefill_bf16_many_tiny_prompts(hd):
     tiles; a few longer prompts in between (several tiles, several token chunks)."""
     shape = fi.ModelShape(2, 256, 8, 2, hd, 512, 2048, 500000.0)
     lens = [1, 2, 3, 1, 1, 2, 5, 1, 4, 1, 150, 2, 1, 3, 1, 1, 70, 2, 2, 1, 5, 1, 1, 3, 9, 1, 2, 1, 1, 4] * 2
-    _prefill_case(shape, True, lens, 256, 1, 9, 1, 0.6, 2e-2, {"attn_chunk": 64})
-    _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2)
+    _prefill_case(shape, True, lens, 256, 1, 9, 1, 0.6, 2e-2, {"prefill_tc": 0, "attn_chunk": 64})
+    _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2, {"prefill_tc": 0})
 
 
 @pytest.mark.parametrize("rows,chunk_tokens", [(20, 64), (256, 64), (37, 128), (256, 1024)])
 def test_prefill_bf16_tensor_core_blocks(rows, chunk_tokens):
-    """Attention of prompt chunks on the tcgen05 tensor cores (option `prefill_tc`): blocks of 128/G consecutive
+    """Attention of prompt chunks on the tcgen05 tensor cores (option `prefill_tc`, the default): blocks of 128/G consecutive
     tokens per work item, at chunk heights that cut blocks at odd places, with prompts of 1 .. 300 tokens (blocks of
     every size, sequences that start in the middle of a chunk, several tiles and several token chunks per block)."""
     _prefill_case(SMALL_GQA, True, [33, 90, 5, 1, 2, 7, 8, 9, 300, 16], rows, 2, 8, 1, 0.6, 2e-2,
