@@ -416,9 +416,13 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *                    itself, from the QKV projection's output.
  *   "prefill_pair"   0 = in first_prefill every prompt token has attention work items of its own.  Default 1:
  *                    two consecutive tokens of a sequence share them (up to 4 query heads per KV head).
- *   "prefill_group"  0 = no groups.  Default 1: in first_prefill up to eight consecutive tokens of a sequence (one
+ *   "prefill_group"  0 = no groups.  Default 1 (used when "prefill_tc" is 0): in first_prefill up to eight consecutive tokens of a sequence (one
  *                    block of eight positions) share attention work items, so a prefix's keys/values are staged once
  *                    per eight tokens (up to 4 query heads per KV head; otherwise the pair form or single rows)
+ *   "prefill_tc"     0 = prompt-chunk attention on the mma.sync kernels ("prefill_group" / "prefill_pair" choose the
+ *                    form).  Default 1: causal attention of prompt chunks on the tcgen05 tensor cores, blocks of
+ *                    128 / (query heads per KV head) consecutive tokens per work item (bfloat16 caches, head_dim 64
+ *                    or 128, 1, 2, 3, 4 or 8 query heads per KV head; otherwise the forms below)
  *   "prefill_rows"   prompt tokens per chunk of first_prefill, 1..256 (default 256; never more than max_batch)
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in
