@@ -135,12 +135,13 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     __shared__ int last_s;
     __shared__ uint32_t lead_s[kTcMaxRows / 32];  // bit i = row i starts a block
     __shared__ float xch_s[2][2][128];            // [tile parity][warpgroup][row]: row maxima (sums at the end)
+    __shared__ int32_t t1_s[kTcMaxRows], slab_s[kTcMaxRows];  // row facts: tokens attended over, first slab row
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.x, c = blockIdx.z, Hkv = gridDim.x, S_max = gridDim.z;
     const int Ce = (C + kTok - 1) / kTok * kTok;  // chunk length in whole tiles
     pdl_wait();  // (row facts come from the kernel before this one)
-    auto t1_of = [&](int i) { return (int)(__ldcg(&rowinfo[i]).x & 0xffffffffll); };
-    auto slab_of = [&](int i) { return (int)(__ldcg(&rowinfo[i]).y & 0x7fffffffll); };  // (< 2^31: the tensor map's row count is)
+    auto t1_of = [&](int i) { return t1_s[i]; };
+    auto slab_of = [&](int i) { return slab_s[i]; };  // (< 2^31: the tensor map's row count is)
     // ---- block starts: eight warps' worth of rows, a ballot each
     for (int wbase = warp * 32; wbase < kTcMaxRows; wbase += (kTcThreads / 32) * 32) {
         const int i = wbase + lane;
@@ -148,6 +149,8 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (i < m) {
             const longlong2 a = __ldcg(&rowinfo[i]);
             const int t1 = (int)(a.x & 0xffffffffll);
+            t1_s[i] = t1;
+            slab_s[i] = (int)(a.y & 0x7fffffffll);
             if (i == 0) {
                 st = true;
             } else {
@@ -332,7 +335,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         {   // Q of this block: float32 -> bfloat16 hi/lo, K-major swizzled rows (the previous block's MMAs are done:
             // its last PV was waited for).  Warp w converts rows 16w .. 16w+15.
             const int sw = warp - 2;
-#pragma unroll 8
+#pragma unroll 16
             for (int e = lane; e < 16 * HD / 4; e += 32) {
                 const int rq = sw * 16 + e / (HD / 4), d4 = (e % (HD / 4)) * 4;
                 const int tq = rq / G, gg = rq - tq * G;
