@@ -423,6 +423,10 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *                    form).  Default 1: causal attention of prompt chunks on the tcgen05 tensor cores, blocks of
  *                    128 / (query heads per KV head) consecutive tokens per work item (bfloat16 caches, head_dim 64
  *                    or 128, 1, 2, 3, 4 or 8 query heads per KV head; otherwise the forms below)
+ *   "prefill_slack"  0..16, default 8: that kernel keeps its softmax weights relative to a reference maximum which
+ *                    moves (and the accumulated output is rescaled) only when a tile's maximum exceeds it by more than
+ *                    2^value; 0 = the reference follows the running maximum exactly (the result is the same up to
+ *                    rounding; tests use 0 to exercise the rescaling)
  *   "prefill_rows"   prompt tokens per chunk of first_prefill, 1..256 (default 256; never more than max_batch)
  *   "fuse_swiglu"    0 = gate/up projection writes float32 sums and a separate kernel applies
  *                    silu(gate)*up.  Default 1: the tensor-core gate/up projection applies it in

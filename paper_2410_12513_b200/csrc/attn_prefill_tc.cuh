@@ -112,13 +112,15 @@ struct PrefillTc {
 // rowinfo[i] = (tokens row i attends over incl. itself | batch row << 32, first slab row) from rope_append (mode 0).
 // q: [m][Hq][HD] float32, rotated and pre-scaled.  tmK/tmV: [Hkv*cap_total][HD] bf16, box 64 x 64.  Scratch and
 // outputs as in attn_split_mma (o_part [m][Hq][S_max][HD], ml_part [m][Hq][S_max], ticket [m][Hkv]).
+// slack_log2: how far (base-2 exponent) a tile's maximum may exceed the reference maximum before the reference moves
+// (8 in production; 0 = it follows the running maximum exactly, which exercises the rescaling of O on most tiles).
 template <int HD, int G>
 __global__ void __launch_bounds__(kTcThreads, 1)  // (ten warps: three share a scheduler's registers, 168 each)
 attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const float* q,
                 int64_t cap_total, const longlong2* rowinfo, int m, const int32_t* __restrict__ m_dev, int Hq, int C,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, uint32_t* __restrict__ ticket,
                 float* __restrict__ out, __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo,
-                uint32_t* __restrict__ flags, uint64_t* stamp) {
+                uint32_t* __restrict__ flags, float slack_log2, uint64_t* stamp) {
     const Stamp stamp_guard(stamp);
     using P = PrefillTc<HD, G>;
     constexpr int TQ = P::TQ, kTok = P::kTok, kHalves = P::kHalves, kBox = P::kBox, kHalfBytes = P::kHalfBytes;
@@ -364,7 +366,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // written out and takes the unmasked path
         const int see = live ? min(T1 + tok, t_end) : 0x7fffffff;
         constexpr float kLog2e = 1.4426950408889634f;
-        constexpr float kSlack = 8.f / kLog2e;  // m_ref moves only when a tile's maximum is this far above it
+        const float kSlack = slack_log2 / kLog2e;  // m_ref moves only when a tile's maximum is this far above it
         const uint32_t o_addr = lane_addr + (uint32_t)(kOCol0 + wg * HH);  // this thread's half of the output row
         for (int j = 0; j < n_tiles; ++j) {
             const int jj = tile0 + j, b = jj & 1;

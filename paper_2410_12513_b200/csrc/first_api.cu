@@ -110,6 +110,7 @@ struct first_ctx {
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
     int prefill_group = 1; // prompt chunks: up to eight consecutive tokens share one (takes precedence over pairs)
+    int prefill_slack = 8; // (its reference maximum moves when a tile's maximum exceeds it by more than 2^this)
     int prefill_tc = 1;    // prompt chunks: attention on the tcgen05 tensor cores, blocks of 128/G tokens (takes precedence over groups)
     int prefill_rows = 0;  // rows per prompt chunk (0: 256)
     int tune_pair_rows = 1;
@@ -674,7 +675,7 @@ int launch_attn_mma(first_ctx* c, cudaStream_t st, int m, const void* kc, const 
         return launch_k(c, st, kClsAttn, attn::attn_prefill_tc<HD, G>, dim3(grid.y, (m + TQ - 1) / TQ + 1, grid.x), \
                         dim3(attn::kTcThreads), attn::PrefillTc<HD, G>::kSmem, *tk, *tv, c->q, kv->cap_total,    \
                         c->rowinfo, m, m_dev, d.n_q_heads, C, c->o_part, c->ml_part, c->ticket, out, out_hi,     \
-                        out_lo, c->flags);                                                                       \
+                        out_lo, c->flags, (float)c->prefill_slack);                                              \
     }
     FIRST_ATTN_TC(128, 1) FIRST_ATTN_TC(128, 2) FIRST_ATTN_TC(128, 3) FIRST_ATTN_TC(128, 4) FIRST_ATTN_TC(128, 8)
     FIRST_ATTN_TC(64, 1) FIRST_ATTN_TC(64, 2) FIRST_ATTN_TC(64, 3) FIRST_ATTN_TC(64, 4) FIRST_ATTN_TC(64, 8)
@@ -1369,6 +1370,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "prefill_pair")) c->prefill_pair = value != 0;
     else if (!std::strcmp(name, "prefill_group")) c->prefill_group = value != 0;
     else if (!std::strcmp(name, "prefill_tc")) c->prefill_tc = value != 0;
+    else if (!std::strcmp(name, "prefill_slack")) c->prefill_slack = (int)std::max<int64_t>(0, std::min<int64_t>(value, 16));
     else if (!std::strcmp(name, "prefill_rows")) c->prefill_rows = value > 0 ? (int)value : 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
     else if (!std::strcmp(name, "tc_mt2_min_rows")) c->tc_mt2_min_rows = value > 0 ? (int)value : -1;

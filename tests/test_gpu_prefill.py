@@ -23,12 +23,18 @@ def _ctx(shape, bf16, max_batch, max_tokens, w):
     return FirstContext(shape, BF16 if bf16 else F32, max_batch, max_tokens, gpu_weights(w))
 
 
-def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_tol, options=None, tight=False):
+def _prefill_case(shape, bf16, lens, max_batch, steps, seed, mode, keep_p, rel_tol, options=None, tight=False,
+                  sharpen=(0, 0)):
     """Oracle prefill per sequence -> routers calibrated on its layer inputs -> one first_prefill
     call on the GPU -> everything it leaves behind compared -> `steps` routed decode steps."""
     import torch
     B, L = len(lens), shape.n_layers
     w = fi.make_weights(shape, seed, bf16)
+    if sharpen != (0, 0):  # query / key projections times 2^a / 2^b (exact in bfloat16): attention scores of several units
+        assert bf16
+        for l in range(L):
+            w["wq"][l] = (w["wq"][l] + np.uint16(sharpen[0] << 7)).astype(np.uint16)
+            w["wk"][l] = (w["wk"][l] + np.uint16(sharpen[1] << 7)).astype(np.uint16)
     om = oracle_model(shape, w)
     prompts = [fi.tokens(shape, int(n), seed, f"prompt{b}") for b, n in enumerate(lens)]
     caps = [int(n) + steps + (3 if b == 0 else 0) for b, n in enumerate(lens)]
@@ -187,6 +193,17 @@ def test_prefill_bf16_tensor_core_blocks_many_tiny_prompts(hd):
     lens = [1, 2, 3, 1, 1, 2, 5, 1, 4, 1, 150, 2, 1, 3, 1, 1, 70, 2, 2, 1, 5, 1, 1, 3, 9, 1, 2, 1, 1, 4] * 2
     _prefill_case(shape, True, lens, 256, 1, 9, 1, 0.6, 2e-2, {"attn_chunk": 64, "prefill_tc": 1})
     _prefill_case(shape, True, lens, 64, 1, 9, 0, 0.6, 2e-2, {"prefill_tc": 1})
+
+
+@pytest.mark.parametrize("hd,slack", [(64, 0), (128, 0), (64, 8), (64, 2)])
+def test_prefill_bf16_tensor_core_blocks_moving_maximum(hd, slack):
+    """Attention scores with a spread of several units (query projection x 8, key projection x 4), prompts of
+    several tiles and token chunks: the softmax's reference maximum has to move while outputs are already
+    accumulated.  `prefill_slack` 0 makes it follow the running maximum exactly, so the accumulated output is
+    rescaled on most tiles; 8 is the production setting, 2 in between: all must give the oracle's result."""
+    shape = fi.ModelShape(2, 4 * hd, 4, 2, hd, 512, 1024, 500000.0)
+    _prefill_case(shape, True, [420, 37, 300, 150], 256, 2, 12, 0, 0.6, 2e-2,
+                  {"prefill_slack": slack, "attn_chunk": 256}, sharpen=(3, 2))
 
 
 def test_prefill_bf16_general_kernels_by_option():
