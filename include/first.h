@@ -423,6 +423,9 @@ int first_step_trace(first_ctx *ctx, int32_t max_n, int32_t *cls, uint64_t *t_st
  *                    form).  Default 1: causal attention of prompt chunks on the tcgen05 tensor cores, blocks of
  *                    128 / (query heads per KV head) consecutive tokens per work item (bfloat16 caches, head_dim 64
  *                    or 128, 1, 2, 3, 4 or 8 query heads per KV head; otherwise the forms below)
+ *   "prefill_lo"     0 = the projections of first_prefill's chunks multiply by the bfloat16 hi half of the
+ *                    activations alone (half the tensor work; plain bfloat16-activation accuracy: measured 2.3e-2 of
+ *                    the logit range at 32 layers, outside the 2e-2 bar).  Default 1: hi + lo halves as everywhere
  *   "prefill_slack"  0..16, default 8: that kernel keeps its softmax weights relative to a reference maximum which
  *                    moves (and the accumulated output is rescaled) only when a tile's maximum exceeds it by more than
  *                    2^value; 0 = the reference follows the running maximum exactly (the result is the same up to

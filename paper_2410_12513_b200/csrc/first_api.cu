@@ -110,6 +110,7 @@ struct first_ctx {
     int fuse_rope = 1;  // the tuned attention kernel rotates q and appends the new key/value itself
     int prefill_pair = 1;  // prompt chunks: two consecutive tokens of a sequence share one attention work item
     int prefill_group = 1; // prompt chunks: up to eight consecutive tokens share one (takes precedence over pairs)
+    int prefill_lo = 1;    // 0 = prompt chunks' projections multiply by the bfloat16 hi half of the activations alone
     int prefill_slack = 8; // (its reference maximum moves when a tile's maximum exceeds it by more than 2^this)
     int prefill_tc = 1;    // prompt chunks: attention on the tcgen05 tensor cores, blocks of 128/G tokens (takes precedence over groups)
     int prefill_rows = 0;  // rows per prompt chunk (0: 256)
@@ -1223,9 +1224,12 @@ int first_prefill(first_ctx* c, const int32_t* tokens, const int32_t* cu_seqlens
                                          c->pf_off, c->pf_cap, c->pf_pos, c->pf_len)));
         if ((rc = check_launch(c))) return rc;
         const PrefillHook ph{router_w, router_b, mode, c->pf_score, total, g0};
+        const int lo_rows_saved = c->tc_lo_max_rows;
+        if (!c->prefill_lo) c->tc_lo_max_rows = 0;
         rc = d.dtype == FIRST_DTYPE_BF16
                  ? decode_step_impl<__nv_bfloat16>(c, c->pf_tok, &vkv, nullptr, nullptr, nullptr, st, &ph)
                  : decode_step_impl<float>(c, c->pf_tok, &vkv, nullptr, nullptr, nullptr, st, &ph);
+        c->tc_lo_max_rows = lo_rows_saved;
         if (rc) return rc;
         FIRST_LAUNCH(kClsPrefillAux, (prefill_keep_last<<<rows, 256, 0, st>>>(c->x, c->pf_cu, B, (int)g0, D, c->x_last)));
         if ((rc = check_launch(c))) return rc;
@@ -1370,6 +1374,7 @@ int first_set_option(first_ctx* c, const char* name, int64_t value) {
     else if (!std::strcmp(name, "prefill_pair")) c->prefill_pair = value != 0;
     else if (!std::strcmp(name, "prefill_group")) c->prefill_group = value != 0;
     else if (!std::strcmp(name, "prefill_tc")) c->prefill_tc = value != 0;
+    else if (!std::strcmp(name, "prefill_lo")) c->prefill_lo = value != 0;
     else if (!std::strcmp(name, "prefill_slack")) c->prefill_slack = (int)std::max<int64_t>(0, std::min<int64_t>(value, 16));
     else if (!std::strcmp(name, "prefill_rows")) c->prefill_rows = value > 0 ? (int)value : 0;
     else if (!std::strcmp(name, "tc_lo_max_rows")) c->tc_lo_max_rows = value >= 0 ? (int)value : (1 << 30);
