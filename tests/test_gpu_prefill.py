@@ -206,6 +206,13 @@ def test_prefill_bf16_tensor_core_blocks_moving_maximum(hd, slack):
                   {"prefill_slack": slack, "attn_chunk": 256}, sharpen=(3, 2))
 
 
+def test_prefill_bf16_plain_activations_by_option():
+    """Option `prefill_lo` 0: the prompt chunks' projections use the bfloat16 hi half of the activations alone.  At
+    three layers this stays inside the bars of the default path (at 32 layers of the 8B shape it does not, which is
+    why it is an option); the decode steps that follow use both halves again."""
+    _prefill_case(SMALL_GQA, True, [8, 200, 77, 130, 1], 256, 3, 5, 0, 0.6, 2e-2, {"prefill_lo": 0})
+
+
 def test_prefill_bf16_general_kernels_by_option():
     _prefill_case(SMALL_GQA, True, [33, 90, 5], 32, 2, 6, 1, 0.6, 2e-2, {"attn_simple": 1, "max_gemv_rows": 1024})
 
