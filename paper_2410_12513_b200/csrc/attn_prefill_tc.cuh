@@ -87,6 +87,8 @@ __device__ __forceinline__ void split2_trunc(float x, float y, uint32_t& hi, uin
     lo = __byte_perm(__float_as_uint(xl), __float_as_uint(yl), 0x7632);
 }
 __device__ __forceinline__ void bar_softmax() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// the two warps (one of each warpgroup) that share a tensor-memory lane quadrant: barriers 2..5
+__device__ __forceinline__ void bar_quadrant(int quad) { asm volatile("bar.sync %0, 64;" ::"r"(2 + quad) : "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -395,7 +397,7 @@ attn_prefill_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
             float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             xch_s[b][wg][r] = mx;
-            bar_softmax();
+            bar_quadrant(quad);  // only the partner warp holds the other half of these rows
             mx = fmaxf(mx, xch_s[b][wg ^ 1][r]);  // (written again two tiles on, a barrier later)
             float alpha = 1.f;
             if (m_ref == -INFINITY) {
